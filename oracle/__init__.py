@@ -198,7 +198,7 @@ def step(shape, head: dict, layers: list, caches: list, kv_len: int, vis, pos, t
     nl = len(layers)
     cfg = _cfg(shape, caches[0][0].shape[1], nl)
     lws = (_LayerW * nl)(*[_layer_struct(w) for w in layers])
-    kvs = (_KV * nl)(*[_KV(k.ctypes.data, v.ctypes.data) for k, v in caches])
+    kvs = (_KV * nl)(*[_KV(k.ctypes.data, v.ctypes.data) for k, v in caches[:nl]])
     logits = np.empty((n, shape.vocab), dtype=np.float64)
     amax = np.empty(n, dtype=np.int32)
     hidden = np.empty((n, shape.d_model), dtype=np.float64) if want_hidden else None
