@@ -1,0 +1,191 @@
+/*
+ * ghd - tree-verification step of speculative decoding on one GPU (sm_100a).
+ *
+ * The operation (paper Sec. II-C, "Predict-then-Verify"): a tree of N drafted
+ * token nodes (node 0 = the root, parent[i] < i) sits on top of a KV cache of
+ * length L.  One forward of the decoder stack is run for all N nodes at once;
+ * node i attends to the whole cache plus only its own root-to-i ancestors
+ * (Sec. II-C, Fig. 3: "a token needs to compute relationships only with
+ * certain tokens"); the row argmax of the logits then decides which drafted
+ * tokens are accepted (the longest validated prefix).
+ *
+ * Conventions
+ *   - "dev" pointers are device memory on the context's GPU, "host" pointers
+ *     are ordinary host memory.  The library never allocates or frees device
+ *     memory: every buffer, the workspace included, belongs to the caller and
+ *     must stay alive until the work enqueued on the stream has finished.
+ *   - All calls enqueue work on the stream given to ghd_create and return
+ *     without synchronising, except ghd_sync_status.
+ *   - Every call returns a ghd_status.  Arguments are validated on the host
+ *     before anything is launched; a failing call launches nothing.
+ *   - Storage type T is float (GHD_F32) or IEEE half (GHD_F16, accumulation in
+ *     float).  Matrices are row-major; weights are stored [out][in].
+ *   - One context per stream; a context is not thread-safe.
+ */
+#ifndef GHD_H_
+#define GHD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GHD_MAX_NODES 256
+
+typedef enum ghd_status {
+    GHD_OK = 0,
+    GHD_EINVAL = 1,       /* null pointer or bad scalar argument                     */
+    GHD_ESHAPE = 2,       /* model shape the kernels do not cover                    */
+    GHD_ETREE = 3,        /* parent array / mask is not a valid tree description     */
+    GHD_ENOSPACE = 4,     /* kv_len + n > max_kv_len, or workspace too small         */
+    GHD_ECUDA = 5,        /* a CUDA runtime/driver call failed                       */
+    GHD_ETIMEOUT = 6,     /* a bounded device-side wait gave up (see ghd_sync_status) */
+    GHD_EUNSUPPORTED = 7
+} ghd_status;
+
+typedef enum ghd_dtype { GHD_F32 = 0, GHD_F16 = 1 } ghd_dtype;
+
+/* Knobs for tests and sweeps (ghd_set_option).  0 always means "automatic". */
+typedef enum ghd_option {
+    GHD_OPT_GEMM_PATH = 0,    /* 0 auto, 1 SIMT kernels, 2 tcgen05 kernels (GHD_F16 only)   */
+    GHD_OPT_ATTN_SPLITS = 1,  /* number of KV splits of the attention (>= 1), 0 auto         */
+    GHD_OPT_ATTN_PATH = 2,    /* 0 auto, 1 SIMT kernel, 2 tcgen05 kernel (GHD_F16 only)      */
+    GHD_OPT_GRAPH = 3,        /* ghd_verify_step: 0/1 = launch kernels directly, 2 = replay a
+                                 CUDA graph captured on first use for the same arguments    */
+    GHD_OPT_GEMM_CTAS = 4     /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
+} ghd_option;
+
+/* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary
+ * embedding (rotate-half pairing), SwiGLU MLP, no biases, n_kv_heads == n_heads. */
+typedef struct ghd_model_cfg {
+    int32_t d_model, n_heads, n_kv_heads, d_head, d_ffn, vocab, n_layers;
+    int32_t max_kv_len;   /* rows of every K/V cache                              */
+    int32_t max_nodes;    /* largest tree, <= GHD_MAX_NODES                        */
+    int32_t dtype;        /* ghd_dtype of weights, caches, activations             */
+    float rms_eps;
+    float rope_theta;
+} ghd_model_cfg;
+
+/* dev pointers, storage type T.  wqkv [3*d_model][d_model] (q rows, then k, then v),
+ * wo [d_model][d_model], w_gate_up [2*d_ffn][d_model] (gate rows, then up rows),
+ * w_down [d_model][d_ffn], rms1/rms2 [d_model]. */
+typedef struct ghd_layer_weights {
+    const void *wqkv, *wo, *w_gate_up, *w_down, *rms1, *rms2;
+} ghd_layer_weights;
+
+typedef struct ghd_model_weights {
+    const void *embed;                /* dev T [vocab][d_model]            */
+    const ghd_layer_weights *layers;  /* HOST array [n_layers]             */
+    const void *rms_final;            /* dev T [d_model]                   */
+    const void *lm_head;              /* dev T [vocab][d_model]            */
+} ghd_model_weights;
+
+/* One layer's cache (paper Sec. II-A: decode appends the new K/V).  k, v: dev T
+ * [n_heads][max_kv_len][d_head]; keys are stored already rotated.  A verify call
+ * reads rows [0, len) and writes the N new rows to [len, len + N) in tree order;
+ * it does not change len. */
+typedef struct ghd_kv_layer {
+    void *k, *v;
+    int32_t len;
+} ghd_kv_layer;
+
+/* A built tree.  The caller fills the five dev pointers with buffers of at least
+ * mask: max_nodes * 4 uint64, parent/depth/pos: max_nodes int32,
+ * rope: max_nodes * d_head float; ghd_tree_build / ghd_tree_from_mask fill the
+ * scalars and enqueue the kernel that fills the buffers.
+ *   mask[i * n_words + w] bit b  = 1 iff new node (64 w + b) is visible to node i
+ *                                  (ancestor or i itself), LSB first;
+ *   depth[i] = edges from the root, pos[i] = kv_len + depth[i] (position id);
+ *   rope[i * d_head + 2 t], [.. + 2 t + 1] = cos, sin of pos[i] * theta^(-2 t / d_head). */
+typedef struct ghd_tree {
+    int32_t n, kv_len, n_words, has_parent;
+    uint64_t *mask;
+    int32_t *parent, *depth, *pos;
+    float *rope;
+} ghd_tree;
+
+/* dev struct written by ghd_accept.  nodes[0..n_matched] is the accepted root
+ * path (nodes[0] = 0); tokens[j] = argmax at nodes[j]; n_emitted = n_matched + 1
+ * (the last token is the one the target model adds itself; paper Table I counts
+ * n_emitted: width 1 gives acceptance length 1). */
+typedef struct ghd_accept_result {
+    int32_t n_matched, n_emitted;
+    int32_t nodes[GHD_MAX_NODES];
+    int32_t tokens[GHD_MAX_NODES];
+} ghd_accept_result;
+
+typedef struct ghd_ctx ghd_ctx;
+
+/* Creates a context bound to `cuda_stream` (a cudaStream_t; NULL = default stream)
+ * on the current device.  GHD_ESHAPE unless d_model == n_heads * d_head,
+ * n_kv_heads == n_heads, d_head in {64, 128}, d_model % 8 == 0, d_ffn % 8 == 0. */
+ghd_status ghd_create(const ghd_model_cfg *cfg, void *cuda_stream, ghd_ctx **out);
+void ghd_destroy(ghd_ctx *ctx);
+
+/* Bytes of scratch the context needs (for cfg.max_nodes and cfg.max_kv_len). */
+size_t ghd_workspace_bytes(const ghd_ctx *ctx);
+/* Hands the context its scratch (dev, 256-byte aligned, caller-owned) and enqueues
+ * the one-time clearing of the parts that must start at zero. */
+ghd_status ghd_set_workspace(ghd_ctx *ctx, void *dev_ptr, size_t bytes);
+ghd_status ghd_set_option(ghd_ctx *ctx, int32_t option, int32_t value);
+
+/* Sec. II-C / III-C-1 (verification tree): parent_host[n], parent[0] = -1,
+ * 0 <= parent[i] < i.  Fills tree->mask/parent/depth/pos/rope (see ghd_tree).
+ * GHD_ETREE on a bad parent array or n outside [1, max_nodes]; GHD_ENOSPACE if
+ * kv_len + n > max_kv_len. */
+ghd_status ghd_tree_build(ghd_ctx *ctx, const int32_t *parent_host, int32_t n, int32_t kv_len, ghd_tree *tree);
+
+/* Same from an explicit visibility mask (Fig. 3d, lookahead-style patterns):
+ * mask_host [n][ceil(n/64)] packed as in ghd_tree; row i must have bit i set and
+ * no bit above i.  depth_host (may be NULL) gives depth[i]; NULL means
+ * popcount(row i) - 1.  parent_host may be NULL (then ghd_accept is refused). */
+ghd_status ghd_tree_from_mask(ghd_ctx *ctx, const uint64_t *mask_host, const int32_t *depth_host,
+                              const int32_t *parent_host, int32_t n, int32_t kv_len, ghd_tree *tree);
+
+/* Sec. II-B (one Transformer layer: MHA block then MLP block) for all tree nodes:
+ *   h = RMSNorm(x) ; q,k,v = h Wqkv^T ; RoPE(q,k) ; K/V rows -> cache[len + i] ;
+ *   o_i = softmax(q_i K_S^T / sqrt(d_head)) V_S over S = cache rows [0,len) plus
+ *   visible new rows (Eq. (1) restricted to the tree) ; y = x + o Wo^T ;
+ *   z = y + (SiLU(h2 Wg^T) * (h2 Wu^T)) Wd^T with h2 = RMSNorm(y).
+ * x_in, x_out: dev T [n][d_model] (may alias).  kv->len must equal tree->kv_len. */
+ghd_status ghd_verify_layer(ghd_ctx *ctx, const ghd_layer_weights *w, ghd_kv_layer *kv, const ghd_tree *tree,
+                            const void *x_in, void *x_out);
+
+/* The whole verify forward: embedding rows of tokens_dev[n], cfg.n_layers layers
+ * (kv[l] is layer l's cache, HOST array), final RMSNorm, lm_head, row argmax
+ * (first index among equal maxima).  logits_dev: float [n][vocab] or NULL (then
+ * the logits live only in the workspace); argmax_dev: int32 [n]. */
+ghd_status ghd_verify_step(ghd_ctx *ctx, const ghd_model_weights *w, ghd_kv_layer *kv, const ghd_tree *tree,
+                           const int32_t *tokens_dev, float *logits_dev, int32_t *argmax_dev);
+
+/* Greedy acceptance (Sec. II-C: fall back to the longest validated prefix): node
+ * c is valid iff every edge (p -> c') on its root path has tokens[c'] == argmax[p];
+ * the deepest valid node wins (lowest index among equals).  out_dev: dev struct. */
+ghd_status ghd_accept(ghd_ctx *ctx, const ghd_tree *tree, const int32_t *tokens_dev, const int32_t *argmax_dev,
+                      ghd_accept_result *out_dev);
+
+/* Building blocks of the layer, exposed for unit tests (same kernels the layer uses).
+ * ghd_linear: y float [n][m] = x T[n][k] * w T[m][k]^T.
+ * ghd_rmsnorm: out T [n][d_model] = RMSNorm(x float [n][d_model]) * g.
+ * ghd_tree_attention: q T [n][n_heads*d_head] (rotated), caches already holding the
+ *   n new rows at [kv_len, kv_len+n) -> out T [n][n_heads*d_head].
+ * ghd_argmax: float [n][v] -> int32 [n]. */
+ghd_status ghd_linear(ghd_ctx *ctx, const void *x, const void *w, int32_t n, int32_t k, int32_t m, float *y);
+ghd_status ghd_rmsnorm(ghd_ctx *ctx, const float *x, const void *g, int32_t n, void *out);
+ghd_status ghd_tree_attention(ghd_ctx *ctx, const void *q, const ghd_kv_layer *kv, const ghd_tree *tree, void *out);
+ghd_status ghd_argmax(ghd_ctx *ctx, const float *logits, int32_t n, int32_t v, int32_t *out);
+
+/* Synchronises the stream and returns GHD_OK, GHD_ECUDA (with the CUDA error kept
+ * for ghd_last_error) or GHD_ETIMEOUT when a kernel's bounded wait expired. */
+ghd_status ghd_sync_status(ghd_ctx *ctx);
+const char *ghd_status_str(ghd_status s);
+const char *ghd_last_error(const ghd_ctx *ctx);
+/* Kernels this context has launched so far (for launch accounting in benchmarks). */
+int64_t ghd_launch_count(const ghd_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GHD_H_ */

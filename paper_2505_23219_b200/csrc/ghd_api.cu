@@ -1,0 +1,385 @@
+// C-ABI entry points of libghd: argument validation, workspace layout, and the
+// order in which the kernels of a layer / a step are enqueued.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+namespace ghd {
+
+struct StepGraph {
+    std::vector<uint64_t> key;
+    cudaGraphExec_t exec;
+    int64_t kernels;
+};
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t carve_workspace(ghd_ctx* c, char* base) {
+    const ghd_model_cfg& m = c->cfg;
+    const size_t N = m.max_nodes, d = m.d_model, f = m.d_ffn, es = (m.dtype == GHD_F32) ? 4 : 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return base ? base + at : nullptr; };
+    const size_t raw_cols = (3 * d > 2 * f) ? 3 * d : 2 * f;
+    c->status = (int*)take(256);
+    c->counters = (int*)take(sizeof(int) * 4096);
+    c->xres = (float*)take(N * d * 4);
+    c->hbuf = take(N * d * es);
+    c->qbuf = take(N * d * es);
+    c->attnbuf = take(N * d * es);
+    c->ubuf = take(N * f * es);
+    c->raw = (float*)take(N * raw_cols * 4);
+    c->att_o = (float*)take((size_t)c->max_splits * N * d * 4);
+    c->att_ml = (float*)take((size_t)c->max_splits * N * m.n_heads * 2 * 4);
+    c->gemm_part = (float*)take((size_t)c->sm_count * 2 * 256 * 128 * 4);
+    c->logits = (float*)take(N * (size_t)m.vocab * 4);
+    return off;
+}
+
+static ghd_status fail(ghd_ctx* c, ghd_status s, const char* what) {
+    if (c) snprintf(c->err, sizeof(c->err), "%s", what);
+    return s;
+}
+
+static ghd_status check_cuda(ghd_ctx* c, const char* where) {
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return GHD_OK;
+    snprintf(c->err, sizeof(c->err), "%s: %s", where, cudaGetErrorString(e));
+    return GHD_ECUDA;
+}
+
+static ghd_status check_tree(ghd_ctx* c, const ghd_tree* t) {
+    if (!t || !t->mask || !t->depth || !t->pos || !t->rope) return fail(c, GHD_EINVAL, "tree: null pointer");
+    if (t->n < 1 || t->n > c->cfg.max_nodes || t->n_words != (t->n + 63) / 64) return fail(c, GHD_ETREE, "tree: not built");
+    if (t->kv_len < 0 || t->kv_len + t->n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: kv_len + n > max_kv_len");
+    return GHD_OK;
+}
+
+// One projection: tcgen05 kernel with the fused epilogue when it applies, else the
+// CUDA-core GEMM into the raw buffer followed by the matching element-wise kernel.
+static ghd_status project(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi,
+                          const ghd_tree* t, const ghd_kv_layer* kv) {
+    const bool tc_ok = c->cfg.dtype == GHD_F16 && gemm_tc_supported(c, n, k, m, epi.mode);
+    if (c->opt_gemm_path == 2 && !tc_ok) return fail(c, GHD_EUNSUPPORTED, "tcgen05 GEMM does not take this shape/type");
+    if (tc_ok && c->opt_gemm_path != 1) return launch_gemm_tc(c, x, w, n, k, m, epi);
+    float* dst = (epi.mode == EPI_RAW) ? epi.out_f32 : c->raw;
+    launch_gemm_simt(c, x, w, n, k, m, dst);
+    switch (epi.mode) {
+        case EPI_ROPE_KV: launch_rope_append(c, dst, t, kv); break;
+        case EPI_RESID: launch_residual(c, dst, n); break;
+        case EPI_SWIGLU: launch_swiglu(c, dst, n); break;
+        default: break;
+    }
+    return GHD_OK;
+}
+
+static ghd_status attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
+    if (c->opt_attn_path == 2) return fail(c, GHD_EUNSUPPORTED, "tcgen05 attention is not built");
+    launch_attn_simt(c, q, kv, t, out);
+    return GHD_OK;
+}
+
+static ghd_status layer_body(ghd_ctx* c, const ghd_layer_weights* w, const ghd_kv_layer* kv, const ghd_tree* t) {
+    const ghd_model_cfg& m = c->cfg;
+    const int n = t->n, d = m.d_model, f = m.d_ffn;
+    ghd_status s;
+    EpiArgs e{};
+    e.rope = t->rope; e.kv_len = t->kv_len; e.max_kv_len = m.max_kv_len; e.d_head = m.d_head; e.d_model = d;
+    launch_rmsnorm(c, c->xres, w->rms1, n, c->hbuf);
+    e.mode = EPI_ROPE_KV; e.out_t = c->qbuf; e.k_cache = kv->k; e.v_cache = kv->v;
+    if ((s = project(c, c->hbuf, w->wqkv, n, d, 3 * d, e, t, kv)) != GHD_OK) return s;
+    if ((s = attention(c, c->qbuf, kv, t, c->attnbuf)) != GHD_OK) return s;
+    e.mode = EPI_RESID; e.out_f32 = c->xres;
+    if ((s = project(c, c->attnbuf, w->wo, n, d, d, e, t, kv)) != GHD_OK) return s;
+    launch_rmsnorm(c, c->xres, w->rms2, n, c->hbuf);
+    e.mode = EPI_SWIGLU; e.out_t = c->ubuf;
+    if ((s = project(c, c->hbuf, w->w_gate_up, n, d, 2 * f, e, t, kv)) != GHD_OK) return s;
+    e.mode = EPI_RESID; e.out_f32 = c->xres;
+    if ((s = project(c, c->ubuf, w->w_down, n, f, d, e, t, kv)) != GHD_OK) return s;
+    return GHD_OK;
+}
+
+static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer* kv, const ghd_tree* t,
+                            const int32_t* tokens, float* logits, int32_t* amax) {
+    const ghd_model_cfg& m = c->cfg;
+    ghd_status s;
+    launch_embed(c, w->embed, tokens, t->n);
+    for (int l = 0; l < m.n_layers; ++l)
+        if ((s = layer_body(c, &w->layers[l], &kv[l], t)) != GHD_OK) return s;
+    launch_rmsnorm(c, c->xres, w->rms_final, t->n, c->hbuf);
+    EpiArgs e{};
+    e.mode = EPI_RAW; e.out_f32 = logits;
+    if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
+    launch_argmax(c, logits, t->n, m.vocab, amax);
+    return GHD_OK;
+}
+
+}  // namespace ghd
+
+using namespace ghd;
+
+extern "C" {
+
+ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out) {
+    if (!cfg || !out) return GHD_EINVAL;
+    *out = nullptr;
+    if (cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->d_ffn <= 0 || cfg->vocab <= 0 || cfg->n_layers < 0 ||
+        cfg->max_kv_len <= 0 || cfg->max_nodes < 1 || cfg->max_nodes > GHD_MAX_NODES ||
+        (cfg->dtype != GHD_F32 && cfg->dtype != GHD_F16) || !(cfg->rms_eps >= 0.f) || !(cfg->rope_theta > 0.f))
+        return GHD_EINVAL;
+    if (cfg->d_model != cfg->n_heads * cfg->d_head || cfg->n_kv_heads != cfg->n_heads ||
+        (cfg->d_head != 64 && cfg->d_head != 128) || cfg->d_model % 8 || cfg->d_ffn % 8)
+        return GHD_ESHAPE;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GHD_ECUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GHD_ECUDA;
+    ghd_ctx* c = new (std::nothrow) ghd_ctx();
+    if (!c) return GHD_EINVAL;
+    memset(c->err, 0, sizeof(c->err));
+    c->cfg = *cfg;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->device = dev;
+    c->sm_count = sms;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = 0;
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+    c->max_splits = 16;
+    c->launches = 0;
+    c->tmaps = new std::map<TmapKey, std::vector<uint64_t>>();
+    c->graphs = new std::vector<StepGraph*>();
+    carve_workspace(c, nullptr);
+    *out = c;
+    return GHD_OK;
+}
+
+void ghd_destroy(ghd_ctx* c) {
+    if (!c) return;
+    for (StepGraph* g : *c->graphs) { cudaGraphExecDestroy(g->exec); delete g; }
+    delete c->graphs;
+    delete c->tmaps;
+    delete c;
+}
+
+size_t ghd_workspace_bytes(const ghd_ctx* c) {
+    if (!c) return 0;
+    ghd_ctx tmp = *c;
+    return carve_workspace(&tmp, nullptr);
+}
+
+ghd_status ghd_set_workspace(ghd_ctx* c, void* dev_ptr, size_t bytes) {
+    if (!c || !dev_ptr) return GHD_EINVAL;
+    if (((uintptr_t)dev_ptr & 255) != 0) return fail(c, GHD_EINVAL, "workspace must be 256-byte aligned");
+    if (bytes < ghd_workspace_bytes(c)) return fail(c, GHD_ENOSPACE, "workspace too small");
+    c->ws = (char*)dev_ptr;
+    c->ws_bytes = bytes;
+    carve_workspace(c, c->ws);
+    // status word and tile arrival counters must start at zero
+    if (cudaMemsetAsync(c->status, 0, 256 + sizeof(int) * 4096, c->stream) != cudaSuccess) return check_cuda(c, "workspace clear");
+    return GHD_OK;
+}
+
+ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
+    if (!c || value < 0) return GHD_EINVAL;
+    switch (option) {
+        case GHD_OPT_GEMM_PATH: if (value > 2) return GHD_EINVAL; c->opt_gemm_path = value; break;
+        case GHD_OPT_ATTN_SPLITS: if (value > c->max_splits) return GHD_EINVAL; c->opt_attn_splits = value; break;
+        case GHD_OPT_ATTN_PATH: if (value > 2) return GHD_EINVAL; c->opt_attn_path = value; break;
+        case GHD_OPT_GRAPH: if (value > 2) return GHD_EINVAL; c->opt_graph = value; break;
+        case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
+        default: return GHD_EINVAL;
+    }
+    return GHD_OK;
+}
+
+static ghd_status tree_common(ghd_ctx* c, int32_t n, int32_t kv_len, ghd_tree* tree) {
+    if (!c || !tree) return GHD_EINVAL;
+    if (!tree->mask || !tree->parent || !tree->depth || !tree->pos || !tree->rope) return fail(c, GHD_EINVAL, "tree: null buffer");
+    if (n < 1 || n > c->cfg.max_nodes) return fail(c, GHD_ETREE, "tree: n outside [1, max_nodes]");
+    if (kv_len < 0) return fail(c, GHD_EINVAL, "tree: negative kv_len");
+    if ((int64_t)kv_len + n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: kv_len + n > max_kv_len");
+    return GHD_OK;
+}
+
+ghd_status ghd_tree_build(ghd_ctx* c, const int32_t* parent_host, int32_t n, int32_t kv_len, ghd_tree* tree) {
+    ghd_status s = tree_common(c, n, kv_len, tree);
+    if (s != GHD_OK) return s;
+    if (!parent_host) return fail(c, GHD_EINVAL, "tree: null parent array");
+    if (parent_host[0] != -1) return fail(c, GHD_ETREE, "tree: parent[0] must be -1");
+    for (int i = 1; i < n; ++i)
+        if (parent_host[i] < 0 || parent_host[i] >= i) return fail(c, GHD_ETREE, "tree: need 0 <= parent[i] < i");
+    tree->n = n; tree->kv_len = kv_len; tree->n_words = (n + 63) / 64; tree->has_parent = 1;
+    launch_tree_build(c, parent_host, tree);
+    return check_cuda(c, "tree_build");
+}
+
+ghd_status ghd_tree_from_mask(ghd_ctx* c, const uint64_t* mask_host, const int32_t* depth_host,
+                              const int32_t* parent_host, int32_t n, int32_t kv_len, ghd_tree* tree) {
+    ghd_status s = tree_common(c, n, kv_len, tree);
+    if (s != GHD_OK) return s;
+    if (!mask_host) return fail(c, GHD_EINVAL, "tree: null mask");
+    const int W = (n + 63) / 64;
+    for (int i = 0; i < n; ++i) {
+        if (!((mask_host[(size_t)i * W + (i >> 6)] >> (i & 63)) & 1ull)) return fail(c, GHD_ETREE, "mask: row lacks its own bit");
+        for (int j = i + 1; j < W * 64; ++j)
+            if ((mask_host[(size_t)i * W + (j >> 6)] >> (j & 63)) & 1ull) return fail(c, GHD_ETREE, "mask: bit above the diagonal");
+        if (depth_host && (depth_host[i] < 0 || depth_host[i] >= n)) return fail(c, GHD_ETREE, "mask: bad depth");
+    }
+    if (parent_host) {
+        if (parent_host[0] != -1) return fail(c, GHD_ETREE, "tree: parent[0] must be -1");
+        for (int i = 1; i < n; ++i)
+            if (parent_host[i] < 0 || parent_host[i] >= i) return fail(c, GHD_ETREE, "tree: need 0 <= parent[i] < i");
+    }
+    tree->n = n; tree->kv_len = kv_len; tree->n_words = W; tree->has_parent = parent_host ? 1 : 0;
+    // pageable host memory: the copies are staged before the call returns
+    cudaMemcpyAsync(tree->mask, mask_host, sizeof(uint64_t) * n * W, cudaMemcpyHostToDevice, c->stream);
+    if (depth_host) cudaMemcpyAsync(tree->depth, depth_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream);
+    if (parent_host) cudaMemcpyAsync(tree->parent, parent_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream);
+    launch_tree_from_mask(c, tree, depth_host != nullptr);
+    return check_cuda(c, "tree_from_mask");
+}
+
+ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer* kv, const ghd_tree* tree,
+                            const void* x_in, void* x_out) {
+    if (!c || !w || !kv || !x_in || !x_out) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (!w->wqkv || !w->wo || !w->w_gate_up || !w->w_down || !w->rms1 || !w->rms2 || !kv->k || !kv->v)
+        return fail(c, GHD_EINVAL, "layer: null weight or cache pointer");
+    ghd_status s = check_tree(c, tree);
+    if (s != GHD_OK) return s;
+    if (kv->len != tree->kv_len) return fail(c, GHD_EINVAL, "layer: kv.len differs from tree.kv_len");
+    launch_load_x(c, x_in, tree->n);
+    if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
+    launch_store_x(c, x_out, tree->n);
+    return check_cuda(c, "verify_layer");
+}
+
+ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer* kv, const ghd_tree* tree,
+                           const int32_t* tokens_dev, float* logits_dev, int32_t* argmax_dev) {
+    if (!c || !w || !kv || !tokens_dev || !argmax_dev) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (!w->embed || !w->rms_final || !w->lm_head || (c->cfg.n_layers > 0 && !w->layers))
+        return fail(c, GHD_EINVAL, "step: null weight pointer");
+    ghd_status s = check_tree(c, tree);
+    if (s != GHD_OK) return s;
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        const ghd_layer_weights& lw = w->layers[l];
+        if (!lw.wqkv || !lw.wo || !lw.w_gate_up || !lw.w_down || !lw.rms1 || !lw.rms2 || !kv[l].k || !kv[l].v)
+            return fail(c, GHD_EINVAL, "step: null layer weight or cache pointer");
+        if (kv[l].len != tree->kv_len) return fail(c, GHD_EINVAL, "step: kv.len differs from tree.kv_len");
+    }
+    float* logits = logits_dev ? logits_dev : c->logits;
+    if (c->opt_graph != 2) {
+        if ((s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev)) != GHD_OK) return s;
+        return check_cuda(c, "verify_step");
+    }
+    // Graph replay: the key is every value the enqueued kernels depend on.
+    std::vector<uint64_t> key;
+    auto push = [&](const void* p) { key.push_back((uint64_t)(uintptr_t)p); };
+    push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
+    push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope);
+    key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
+    key.push_back(((uint64_t)(uint32_t)c->opt_gemm_path << 48) | ((uint64_t)(uint32_t)c->opt_attn_splits << 32) |
+                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | (uint32_t)c->opt_gemm_ctas);
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        const ghd_layer_weights& lw = w->layers[l];
+        push(lw.wqkv); push(lw.wo); push(lw.w_gate_up); push(lw.w_down); push(lw.rms1); push(lw.rms2);
+        push(kv[l].k); push(kv[l].v);
+    }
+    for (StepGraph* g : *c->graphs)
+        if (g->key == key) {
+            if (cudaGraphLaunch(g->exec, c->stream) != cudaSuccess) return check_cuda(c, "graph launch");
+            c->launches += g->kernels;
+            return GHD_OK;
+        }
+    const int64_t before = c->launches;
+    if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return check_cuda(c, "begin capture");
+    s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(c->stream, &graph);
+    if (s != GHD_OK) { if (graph) cudaGraphDestroy(graph); c->launches = before; return s; }
+    if (ce != cudaSuccess || !graph) { c->launches = before; cudaGetLastError(); return fail(c, GHD_ECUDA, "stream capture failed"); }
+    cudaGraphExec_t exec = nullptr;
+    if (cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) { cudaGraphDestroy(graph); c->launches = before; return check_cuda(c, "graph instantiate"); }
+    cudaGraphDestroy(graph);
+    StepGraph* g = new StepGraph{key, exec, c->launches - before};
+    if (c->graphs->size() >= 8) { cudaGraphExecDestroy(c->graphs->front()->exec); delete c->graphs->front(); c->graphs->erase(c->graphs->begin()); }
+    c->graphs->push_back(g);
+    if (cudaGraphLaunch(exec, c->stream) != cudaSuccess) return check_cuda(c, "graph launch");
+    return GHD_OK;
+}
+
+ghd_status ghd_accept(ghd_ctx* c, const ghd_tree* tree, const int32_t* tokens_dev, const int32_t* argmax_dev,
+                      ghd_accept_result* out_dev) {
+    if (!c || !tokens_dev || !argmax_dev || !out_dev) return GHD_EINVAL;
+    ghd_status s = check_tree(c, tree);
+    if (s != GHD_OK) return s;
+    if (!tree->has_parent || !tree->parent) return fail(c, GHD_EINVAL, "accept: tree has no parent array");
+    launch_accept(c, tree, tokens_dev, argmax_dev, out_dev);
+    return check_cuda(c, "accept");
+}
+
+ghd_status ghd_linear(ghd_ctx* c, const void* x, const void* w, int32_t n, int32_t k, int32_t m, float* y) {
+    if (!c || !x || !w || !y || n < 1 || k < 1 || m < 1) return GHD_EINVAL;
+    if (n > c->cfg.max_nodes) return fail(c, GHD_ENOSPACE, "linear: n > max_nodes");
+    if (k % 8) return fail(c, GHD_ESHAPE, "linear: k must be a multiple of 8");
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    EpiArgs e{};
+    e.mode = EPI_RAW; e.out_f32 = y;
+    ghd_status s = project(c, x, w, n, k, m, e, nullptr, nullptr);
+    return s != GHD_OK ? s : check_cuda(c, "linear");
+}
+
+ghd_status ghd_rmsnorm(ghd_ctx* c, const float* x, const void* g, int32_t n, void* out) {
+    if (!c || !x || !g || !out || n < 1) return GHD_EINVAL;
+    launch_rmsnorm(c, x, g, n, out);
+    return check_cuda(c, "rmsnorm");
+}
+
+ghd_status ghd_tree_attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* tree, void* out) {
+    if (!c || !q || !kv || !kv->k || !kv->v || !out) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    ghd_status s = check_tree(c, tree);
+    if (s != GHD_OK) return s;
+    if ((s = attention(c, q, kv, tree, out)) != GHD_OK) return s;
+    return check_cuda(c, "tree_attention");
+}
+
+ghd_status ghd_argmax(ghd_ctx* c, const float* logits, int32_t n, int32_t v, int32_t* out) {
+    if (!c || !logits || !out || n < 1 || v < 1) return GHD_EINVAL;
+    launch_argmax(c, logits, n, v, out);
+    return check_cuda(c, "argmax");
+}
+
+ghd_status ghd_sync_status(ghd_ctx* c) {
+    if (!c) return GHD_EINVAL;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return check_cuda(c, "stream synchronize");
+    if (!c->ws) return GHD_OK;
+    int st = 0;
+    if (cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return check_cuda(c, "status read");
+    if (st != DEV_OK) {
+        snprintf(c->err, sizeof(c->err), "device wait expired (code %d)", st);
+        cudaMemset(c->status, 0, sizeof(int));
+        return GHD_ETIMEOUT;
+    }
+    return GHD_OK;
+}
+
+const char* ghd_status_str(ghd_status s) {
+    switch (s) {
+        case GHD_OK: return "ok";
+        case GHD_EINVAL: return "invalid argument";
+        case GHD_ESHAPE: return "unsupported model shape";
+        case GHD_ETREE: return "invalid tree";
+        case GHD_ENOSPACE: return "not enough space";
+        case GHD_ECUDA: return "CUDA error";
+        case GHD_ETIMEOUT: return "device wait timed out";
+        case GHD_EUNSUPPORTED: return "unsupported";
+    }
+    return "unknown";
+}
+
+const char* ghd_last_error(const ghd_ctx* c) { return c ? c->err : ""; }
+int64_t ghd_launch_count(const ghd_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,105 @@
+// Internal declarations shared by the translation units of libghd.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <tuple>
+#include <vector>
+
+#include "ghd.h"
+
+namespace ghd {
+
+// Device status word values (first failure wins).
+enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_TIMEOUT_TMEM = 4 };
+
+// Epilogues of the projection GEMMs.
+enum Epilogue : int {
+    EPI_RAW = 0,      // out float [n][m] = acc
+    EPI_ROPE_KV = 1,  // q rotated -> q buffer; k rotated, v -> cache rows kv_len + i
+    EPI_RESID = 2,    // xres[n][m] += acc (float residual stream)
+    EPI_SWIGLU = 3,   // u T [n][m/2] = SiLU(gate) * up, weight rows [gate | up]
+};
+
+struct EpiArgs {
+    int mode;
+    float* out_f32;       // EPI_RAW target / EPI_RESID residual stream (in place)
+    void* out_t;          // EPI_ROPE_KV: q buffer T [n][d]; EPI_SWIGLU: u T [n][f]
+    void* k_cache;        // EPI_ROPE_KV
+    void* v_cache;
+    const float* rope;    // [n][d_head] cos/sin pairs
+    int kv_len, max_kv_len, d_head, d_model;
+};
+
+struct TmapKey {
+    const void* ptr; uint64_t rows, cols; uint32_t box_rows, box_cols;
+    bool operator<(const TmapKey& o) const {
+        return std::tie(ptr, rows, cols, box_rows, box_cols) < std::tie(o.ptr, o.rows, o.cols, o.box_rows, o.box_cols);
+    }
+};
+
+struct StepGraph;
+
+}  // namespace ghd
+
+struct ghd_ctx {
+    ghd_model_cfg cfg;
+    cudaStream_t stream;
+    int device, sm_count;
+    // options
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas;
+    // workspace carve (all device pointers into the caller's buffer)
+    char* ws;
+    size_t ws_bytes;
+    float* xres;      // [max_nodes][d_model] residual stream
+    void* hbuf;       // T [max_nodes][d_model] normalised activations
+    void* qbuf;       // T [max_nodes][d_model] rotated queries
+    void* attnbuf;    // T [max_nodes][d_model] attention output
+    void* ubuf;       // T [max_nodes][d_ffn]
+    float* raw;       // float [max_nodes][max(3 d_model, 2 d_ffn)] un-fused GEMM output
+    float* att_o;     // float [splits][max_nodes][d_model] attention partial numerators
+    float* att_ml;    // float [splits][max_nodes][n_heads][2] running max / sum
+    float* gemm_part; // float [ctas][2][256][128] split tile partial sums
+    int* counters;    // int [tiles] arrival counters (zero between launches)
+    float* logits;    // float [max_nodes][vocab]
+    int* status;      // device status word
+    int max_splits;
+    // bookkeeping
+    int64_t launches;
+    char err[256];
+    std::map<ghd::TmapKey, std::vector<uint64_t>>* tmaps;   // cached tensor maps (128-byte blobs)
+    std::vector<ghd::StepGraph*>* graphs;
+};
+
+namespace ghd {
+
+size_t carve_workspace(ghd_ctx* c, char* base);   // returns bytes needed; assigns pointers when base != nullptr
+
+// kernels_small.cu
+void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t);
+void launch_tree_from_mask(ghd_ctx* c, const ghd_tree* t, bool have_depth);   // mask/depth already copied
+void launch_load_x(ghd_ctx* c, const void* x_in, int n);     // T [n][d] -> xres
+void launch_store_x(ghd_ctx* c, void* x_out, int n);         // xres -> T [n][d]
+void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n);
+void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out);
+void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, const ghd_kv_layer* kv);
+void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n);
+void launch_residual(ghd_ctx* c, const float* proj_raw, int n);
+void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out);
+void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out);
+
+// gemm_simt.cu : y float [n][m] = x T [n][k] * w T [m][k]^T
+void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, float* y);
+
+// attn_simt.cu : split-KV tree attention + combine
+void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
+int attn_auto_splits(const ghd_ctx* c, int n, int kv_total);
+
+// gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
+ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
+bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode);
+
+}  // namespace ghd

@@ -1,0 +1,326 @@
+// Small kernels of the verify step: tree build, embedding gather, RMSNorm,
+// RoPE + KV append, SwiGLU, residual add, row argmax, acceptance walk.
+#include "internal.h"
+
+namespace ghd {
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+
+#define GHD_DISPATCH_T(c, expr_f32, expr_f16) \
+    do { if ((c)->cfg.dtype == GHD_F32) { expr_f32; } else { expr_f16; } } while (0)
+
+// ---------------------------------------------------------------- tree build
+struct ParentArg { int16_t p[GHD_MAX_NODES]; };
+
+// Thread i walks from node i to the root, setting one mask bit per ancestor.
+// The rotary table is computed in double so that the angle pos * theta^(-2t/dh)
+// carries no float rounding of the frequency.
+__global__ void k_tree_build(ParentArg pa, int n, int n_words, int kv_len, int d_head, double theta,
+                             uint64_t* mask, int32_t* parent, int32_t* depth, int32_t* pos, float* rope) {
+    const int i = threadIdx.x;
+    if (i < n) {
+        uint64_t row[GHD_MAX_NODES / 64] = {0, 0, 0, 0};
+        int steps = 0;
+        for (int a = i; a >= 0 && steps <= n; a = pa.p[a]) { row[a >> 6] |= 1ull << (a & 63); ++steps; }
+        for (int w = 0; w < n_words; ++w) mask[i * n_words + w] = row[w];
+        parent[i] = pa.p[i];
+        depth[i] = steps - 1;
+        pos[i] = kv_len + steps - 1;
+    }
+    __syncthreads();
+    const int half = d_head / 2;
+    for (int e = threadIdx.x; e < n * half; e += blockDim.x) {
+        const int node = e / half, t = e % half;
+        const double ang = (double)pos[node] * pow(theta, -2.0 * t / d_head);
+        double s, c;
+        sincos(ang, &s, &c);
+        rope[node * d_head + 2 * t] = (float)c;
+        rope[node * d_head + 2 * t + 1] = (float)s;
+    }
+}
+
+// Explicit-mask variant: mask (and optionally depth, parent) were copied in.
+__global__ void k_tree_from_mask(int n, int n_words, int kv_len, int d_head, double theta, int have_depth,
+                                 const uint64_t* mask, int32_t* depth, int32_t* pos, float* rope) {
+    const int i = threadIdx.x;
+    if (i < n) {
+        int dep;
+        if (have_depth) dep = depth[i];
+        else {
+            int bits = 0;
+            for (int w = 0; w < n_words; ++w) bits += __popcll(mask[i * n_words + w]);
+            dep = bits - 1;
+            depth[i] = dep;
+        }
+        pos[i] = kv_len + dep;
+    }
+    __syncthreads();
+    const int half = d_head / 2;
+    for (int e = threadIdx.x; e < n * half; e += blockDim.x) {
+        const int node = e / half, t = e % half;
+        const double ang = (double)pos[node] * pow(theta, -2.0 * t / d_head);
+        double s, c;
+        sincos(ang, &s, &c);
+        rope[node * d_head + 2 * t] = (float)c;
+        rope[node * d_head + 2 * t + 1] = (float)s;
+    }
+}
+
+void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t) {
+    ParentArg pa;
+    for (int i = 0; i < GHD_MAX_NODES; ++i) pa.p[i] = (int16_t)(i < t->n ? parent_host[i] : -1);
+    k_tree_build<<<1, GHD_MAX_NODES, 0, c->stream>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
+                                                     (double)c->cfg.rope_theta, t->mask, t->parent, t->depth,
+                                                     t->pos, t->rope);
+    c->launches++;
+}
+
+void launch_tree_from_mask(ghd_ctx* c, const ghd_tree* t, bool have_depth) {
+    k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->stream>>>(t->n, t->n_words, t->kv_len, c->cfg.d_head,
+                                                         (double)c->cfg.rope_theta, have_depth ? 1 : 0, t->mask,
+                                                         t->depth, t->pos, t->rope);
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- x in / out, embedding
+template <typename T>
+__global__ void k_load_x(const T* __restrict__ x, float* __restrict__ xres, size_t count) {
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x)
+        xres[e] = to_f32<T>(x[e]);
+}
+
+template <typename T>
+__global__ void k_store_x(const float* __restrict__ xres, T* __restrict__ x, size_t count) {
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x)
+        x[e] = from_f32<T>(xres[e]);
+}
+
+template <typename T>
+__global__ void k_embed(const T* __restrict__ table, const int32_t* __restrict__ tokens, float* __restrict__ xres, int d) {
+    const T* row = table + (size_t)tokens[blockIdx.x] * d;
+    for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x) xres[(size_t)blockIdx.x * d + cidx] = to_f32<T>(row[cidx]);
+}
+
+static int grid_for(size_t count, int block, int cap) {
+    size_t g = (count + block - 1) / block;
+    return (int)(g < 1 ? 1 : (g > (size_t)cap ? cap : g));
+}
+
+void launch_load_x(ghd_ctx* c, const void* x_in, int n) {
+    const size_t count = (size_t)n * c->cfg.d_model;
+    const int g = grid_for(count, 256, 4 * c->sm_count);
+    GHD_DISPATCH_T(c, (k_load_x<float><<<g, 256, 0, c->stream>>>((const float*)x_in, c->xres, count)),
+                   (k_load_x<__half><<<g, 256, 0, c->stream>>>((const __half*)x_in, c->xres, count)));
+    c->launches++;
+}
+
+void launch_store_x(ghd_ctx* c, void* x_out, int n) {
+    const size_t count = (size_t)n * c->cfg.d_model;
+    const int g = grid_for(count, 256, 4 * c->sm_count);
+    GHD_DISPATCH_T(c, (k_store_x<float><<<g, 256, 0, c->stream>>>(c->xres, (float*)x_out, count)),
+                   (k_store_x<__half><<<g, 256, 0, c->stream>>>(c->xres, (__half*)x_out, count)));
+    c->launches++;
+}
+
+void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n) {
+    GHD_DISPATCH_T(c, (k_embed<float><<<n, 256, 0, c->stream>>>((const float*)embed, tokens, c->xres, c->cfg.d_model)),
+                   (k_embed<__half><<<n, 256, 0, c->stream>>>((const __half*)embed, tokens, c->xres, c->cfg.d_model)));
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- RMSNorm
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    if (l == 0) red[w] = v;
+    __syncthreads();
+    const int nw = (blockDim.x + 31) >> 5;
+    float t = (threadIdx.x < nw) ? red[threadIdx.x] : 0.f;
+    if (w == 0) {
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (l == 0) red[0] = t;
+    }
+    __syncthreads();
+    const float r = red[0];
+    __syncthreads();
+    return r;
+}
+
+// One block per row: out = x * g / sqrt(mean(x^2) + eps), math in float.
+template <typename T>
+__global__ void k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, T* __restrict__ out, int d, float eps) {
+    __shared__ float red[32];
+    const float* row = x + (size_t)blockIdx.x * d;
+    float ss = 0.f;
+    for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x) { const float v = row[cidx]; ss += v * v; }
+    ss = block_sum(ss, red);
+    const float r = rsqrtf(ss / (float)d + eps);
+    for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x)
+        out[(size_t)blockIdx.x * d + cidx] = from_f32<T>(row[cidx] * r * to_f32<T>(g[cidx]));
+}
+
+void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out) {
+    const int d = c->cfg.d_model;
+    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, 256, 0, c->stream>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
+                   (k_rmsnorm<__half><<<n, 256, 0, c->stream>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- RoPE + KV append (un-fused path)
+// qkv float [n][3 d].  Thread per (node, head, t < dh/2): rotates the q and k pairs
+// (t, t + dh/2), writes q to the query buffer and k, v to cache row kv_len + node.
+template <typename T>
+__global__ void k_rope_append(const float* __restrict__ qkv, const float* __restrict__ rope, T* __restrict__ q,
+                              T* __restrict__ kc, T* __restrict__ vc, int n, int heads, int dh, int kv_len, int max_kv) {
+    const int half = dh / 2, d = heads * dh;
+    const size_t total = (size_t)n * heads * half;
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const int t = (int)(e % half), h = (int)((e / half) % heads), i = (int)(e / ((size_t)half * heads));
+        const float cs = rope[i * dh + 2 * t], sn = rope[i * dh + 2 * t + 1];
+        const float* base = qkv + (size_t)i * 3 * d + h * dh;
+        const float qa = base[t], qb = base[t + half];
+        const float ka = base[d + t], kb = base[d + t + half];
+        T* qo = q + (size_t)i * d + h * dh;
+        qo[t] = from_f32<T>(qa * cs - qb * sn);
+        qo[t + half] = from_f32<T>(qb * cs + qa * sn);
+        const size_t crow = ((size_t)h * max_kv + kv_len + i) * dh;
+        kc[crow + t] = from_f32<T>(ka * cs - kb * sn);
+        kc[crow + t + half] = from_f32<T>(kb * cs + ka * sn);
+        vc[crow + t] = from_f32<T>(base[2 * d + t]);
+        vc[crow + t + half] = from_f32<T>(base[2 * d + t + half]);
+    }
+}
+
+void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, const ghd_kv_layer* kv) {
+    const ghd_model_cfg& m = c->cfg;
+    const size_t total = (size_t)t->n * m.n_heads * (m.d_head / 2);
+    const int g = grid_for(total, 256, 8 * c->sm_count);
+    GHD_DISPATCH_T(c,
+        (k_rope_append<float><<<g, 256, 0, c->stream>>>(qkv_raw, t->rope, (float*)c->qbuf, (float*)kv->k, (float*)kv->v,
+                                                         t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)),
+        (k_rope_append<__half><<<g, 256, 0, c->stream>>>(qkv_raw, t->rope, (__half*)c->qbuf, (__half*)kv->k, (__half*)kv->v,
+                                                          t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)));
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- SwiGLU, residual (un-fused path)
+template <typename T>
+__global__ void k_swiglu(const float* __restrict__ gu, T* __restrict__ u, int n, int f) {
+    const size_t total = (size_t)n * f;
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const size_t i = e / f, cidx = e % f;
+        const float g = gu[i * 2 * f + cidx], up = gu[i * 2 * f + f + cidx];
+        u[e] = from_f32<T>(g / (1.f + expf(-g)) * up);
+    }
+}
+
+void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n) {
+    const size_t total = (size_t)n * c->cfg.d_ffn;
+    const int g = grid_for(total, 256, 8 * c->sm_count);
+    GHD_DISPATCH_T(c, (k_swiglu<float><<<g, 256, 0, c->stream>>>(gu_raw, (float*)c->ubuf, n, c->cfg.d_ffn)),
+                   (k_swiglu<__half><<<g, 256, 0, c->stream>>>(gu_raw, (__half*)c->ubuf, n, c->cfg.d_ffn)));
+    c->launches++;
+}
+
+__global__ void k_residual(float* __restrict__ xres, const float* __restrict__ proj, size_t count) {
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x)
+        xres[e] += proj[e];
+}
+
+void launch_residual(ghd_ctx* c, const float* proj_raw, int n) {
+    const size_t count = (size_t)n * c->cfg.d_model;
+    k_residual<<<grid_for(count, 256, 8 * c->sm_count), 256, 0, c->stream>>>(c->xres, proj_raw, count);
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- row argmax
+// One block per row; each warp scans a strided slice, lanes keep (value, index)
+// with "greater value, or equal value and smaller index" as the order, so equal
+// maxima resolve to the first index.  NaN never wins.
+__device__ __forceinline__ void amax_merge(float& v, int& i, float ov, int oi) {
+    if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+}
+
+__global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __restrict__ out) {
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    const float* row = logits + (size_t)blockIdx.x * v;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int cidx = threadIdx.x; cidx < v; cidx += blockDim.x) amax_merge(best, bi, row[cidx], cidx);
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        amax_merge(best, bi, ov, oi);
+    }
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    if (l == 0) { sv[w] = best; si[w] = bi; }
+    __syncthreads();
+    if (w == 0) {
+        const int nw = blockDim.x >> 5;
+        best = l < nw ? sv[l] : -INFINITY;
+        bi = l < nw ? si[l] : 0x7fffffff;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            amax_merge(best, bi, ov, oi);
+        }
+        if (l == 0) out[blockIdx.x] = (bi == 0x7fffffff) ? 0 : bi;
+    }
+}
+
+void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out) {
+    k_argmax<<<n, 512, 0, c->stream>>>(logits, v, out);
+    c->launches++;
+}
+
+// ---------------------------------------------------------------- acceptance
+// Thread i checks every edge on the root path of node i; the deepest valid node
+// wins, the lowest index among equally deep ones.  Thread 0 then writes the path.
+__global__ void k_accept(int n, const int32_t* __restrict__ parent,
+                         const int32_t* __restrict__ tokens, const int32_t* __restrict__ amax,
+                         ghd_accept_result* __restrict__ out) {
+    __shared__ int key[GHD_MAX_NODES];
+    const int i = threadIdx.x;
+    int k = -1;
+    if (i < n) {
+        bool ok = true;
+        int dep = 0;
+        for (int cnode = i; cnode > 0 && dep <= n; ++dep) {
+            const int p = parent[cnode];
+            if (tokens[cnode] != amax[p]) ok = false;
+            cnode = p;
+        }
+        if (ok) k = dep * GHD_MAX_NODES + (GHD_MAX_NODES - 1 - i);
+    }
+    key[i] = k;
+    __syncthreads();
+    for (int s = GHD_MAX_NODES / 2; s > 0; s >>= 1) {
+        if (i < s) key[i] = max(key[i], key[i + s]);
+        __syncthreads();
+    }
+    if (i == 0) {
+        const int best = key[0];
+        const int dep = best / GHD_MAX_NODES, win = GHD_MAX_NODES - 1 - (best % GHD_MAX_NODES);
+        out->n_matched = dep;
+        out->n_emitted = dep + 1;
+        int cnode = win;
+        for (int j = dep; j >= 0; --j) {
+            out->nodes[j] = cnode;
+            out->tokens[j] = amax[cnode];
+            cnode = (j > 0) ? parent[cnode] : 0;
+        }
+    }
+}
+
+void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out) {
+    k_accept<<<1, GHD_MAX_NODES, 0, c->stream>>>(t->n, t->parent, tokens, amax, out);
+    c->launches++;
+}
+
+}  // namespace ghd

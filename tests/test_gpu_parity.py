@@ -1,0 +1,331 @@
+"""GPU parity: every call goes through the C-ABI and is compared with the CPU
+oracle on the same seeded inputs.  Integer results bit-exact; floating point
+within max|got-want|/max|want| <= 1e-4 (float mode) or 2e-2 (half mode)."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+from util import (argmax_margin_ok, gpu_cfg, gpu_layer_weights, max_rel_err, to_dev, tol_for, unpack_mask)
+
+pytestmark = pytest.mark.gpu
+
+SMALL32 = wl.scaled(wl.TINY, name="small32", d_model=256, n_heads=4, d_head=64, d_ffn=352, vocab=777, n_layers=2)
+SMALL16 = wl.scaled(SMALL32, name="small16", dtype="f16")
+SMALL16_DH128 = wl.scaled(SMALL16, name="small16b", d_model=512, n_heads=4, d_head=128, d_ffn=704)
+
+
+@pytest.fixture(scope="module")
+def ghd():
+    import paper_2505_23219_b200 as g
+    return g
+
+
+def make_ctx(ghd, shape, max_kv_len, max_nodes, n_layers=None):
+    return ghd.ghd_create(gpu_cfg(shape, max_kv_len, max_nodes, n_layers))
+
+
+# ---------------------------------------------------------------- tree build (bit-exact)
+TREES = [("chain1", wl.chain_tree(1)), ("chain9", wl.chain_tree(9)), ("star33", wl.star_tree(33)),
+         ("medusa64", wl.medusa_tree(64)), ("rand8", wl.random_tree(8, 4, 1)), ("rand63", wl.random_tree(63, 8, 2)),
+         ("rand65", wl.random_tree(65, 8, 3)), ("rand129", wl.random_tree(129, 8, 4)),
+         ("rand256", wl.random_tree(256, 8, 5, max_children=6)), ("chain256", wl.chain_tree(256))]
+
+
+@pytest.mark.parametrize("name,parent", TREES, ids=[t[0] for t in TREES])
+def test_tree_build_bit_exact(ghd, name, parent):
+    ctx = make_ctx(ghd, SMALL32, 1024, 256)
+    kv_len = 300
+    tree = ghd.ghd_tree_build(ctx, parent, kv_len)
+    ghd.ghd_sync_status(ctx)
+    n = len(parent)
+    vis, depth, pos = oracle.tree_build(parent, kv_len)
+    assert tree.c.n == n and tree.c.n_words == (n + 63) // 64
+    assert np.array_equal(unpack_mask(tree.mask_words(), n), vis)
+    assert np.array_equal(tree.depth[:n].cpu().numpy(), depth)
+    assert np.array_equal(tree.pos[:n].cpu().numpy(), pos)
+    assert np.array_equal(tree.parent[:n].cpu().numpy(), np.asarray(parent, dtype=np.int32))
+    # rotary table: cos/sin of pos * theta^(-2t/dh), checked through the oracle's rotation of unit vectors
+    dh = SMALL32.d_head
+    unit = np.zeros((n, 1, dh))
+    unit[:, 0, : dh // 2] = 1.0
+    rot = oracle.rope(unit, pos, SMALL32.rope_theta)[:, 0]
+    table = tree.rope[: n * dh].cpu().numpy().reshape(n, dh // 2, 2)
+    assert np.abs(table[:, :, 0] - rot[:, : dh // 2]).max() < 1e-6
+    assert np.abs(table[:, :, 1] - rot[:, dh // 2:]).max() < 1e-6
+
+
+def test_tree_from_explicit_lookahead_mask_equals_tree_build(ghd):
+    ctx = make_ctx(ghd, SMALL32, 1024, 64)
+    vis, depth, parent = wl.lookahead_pattern(7, 5, 5)
+    a = ghd.ghd_tree_from_mask(ctx, ghd.pack_mask(vis), 100, parent=parent)
+    b = ghd.ghd_tree_build(ctx, parent, 100)
+    c = ghd.ghd_tree_from_mask(ctx, ghd.pack_mask(vis), 100, depth=depth)
+    ghd.ghd_sync_status(ctx)
+    n = len(parent)
+    assert np.array_equal(a.mask_words(), b.mask_words())
+    for t in (a, c):
+        assert np.array_equal(t.depth[:n].cpu().numpy(), b.depth[:n].cpu().numpy())
+        assert np.array_equal(t.pos[:n].cpu().numpy(), b.pos[:n].cpu().numpy())
+        assert np.array_equal(t.rope.cpu().numpy(), b.rope.cpu().numpy())
+    assert np.array_equal(unpack_mask(a.mask_words(), n), vis.astype(np.uint8))
+
+
+def test_argument_errors_launch_nothing(ghd):
+    ctx = make_ctx(ghd, SMALL32, 128, 16)
+    before = ghd.ghd_launch_count(ctx)
+    cases = [([0, 0], 0, "GHD_ETREE"), ([-1, 1], 0, "GHD_ETREE"), ([-1, -1], 0, "GHD_ETREE"),
+             ([-1] + [0] * 16, 0, "GHD_ETREE"), ([], 0, "GHD_ETREE"), ([-1, 0], 127, "GHD_ENOSPACE"),
+             ([-1, 0], -1, "GHD_EINVAL")]
+    for parent, kv_len, want in cases:
+        with pytest.raises(ghd.GhdError) as e:
+            ghd.ghd_tree_build(ctx, parent, kv_len)
+        assert e.value.name == want
+    bad = ghd.pack_mask(np.array([[1, 0], [1, 0]], dtype=bool))          # row 1 lacks its own bit
+    with pytest.raises(ghd.GhdError) as e:
+        ghd.ghd_tree_from_mask(ctx, bad, 0)
+    assert e.value.name == "GHD_ETREE"
+    up = ghd.pack_mask(np.array([[1, 1], [1, 1]], dtype=bool))           # bit above the diagonal
+    with pytest.raises(ghd.GhdError):
+        ghd.ghd_tree_from_mask(ctx, up, 0)
+    assert ghd.ghd_launch_count(ctx) == before
+    with pytest.raises(ghd.GhdError) as e:                               # unsupported shapes
+        ghd.ghd_create(gpu_cfg(wl.scaled(SMALL32, d_head=32, n_heads=8), 128, 16))
+    assert e.value.name == "GHD_ESHAPE"
+    with pytest.raises(ghd.GhdError) as e:
+        ghd.ghd_create(gpu_cfg(SMALL32, 128, 257))
+    assert e.value.name == "GHD_EINVAL"
+    # a tree that was never built is refused by the compute calls
+    tree = ghd.Tree(ctx)
+    with pytest.raises(ghd.GhdError):
+        ghd.ghd_accept(ctx, tree, to_dev(np.zeros(4, np.int32)), to_dev(np.zeros(4, np.int32)))
+    ghd.ghd_sync_status(ctx)
+
+
+# ---------------------------------------------------------------- building blocks
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16], ids=["f32", "f16"])
+@pytest.mark.parametrize("n", [1, 5, 8, 37])
+def test_rmsnorm(ghd, shape, n):
+    ctx = make_ctx(ghd, shape, 128, 64)
+    x = wl.normal((n, shape.d_model), 301, 3.0)
+    g = wl.normal((shape.d_model,), 302, 0.1, 1.0, dtype=shape.dtype)
+    out = ghd.ghd_rmsnorm(ctx, to_dev(x), to_dev(g))
+    ghd.ghd_sync_status(ctx)
+    want = oracle.rmsnorm(x, g, shape.rms_eps)
+    assert max_rel_err(out.cpu().numpy(), want) <= (1e-6 if shape.dtype == "f32" else 1e-3)
+
+
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16], ids=["f32", "f16"])
+@pytest.mark.parametrize("n,k,m", [(1, 256, 40), (7, 352, 256), (8, 256, 1001), (19, 1376, 130), (64, 512, 96)])
+def test_linear_cuda_core_path(ghd, shape, n, k, m):
+    ctx = make_ctx(ghd, shape, 128, 64)
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PATH, 1)
+    x = wl.normal((n, k), 311, 1.0, dtype=shape.dtype)
+    w = wl.normal((m, k), 312, 0.02, dtype=shape.dtype)
+    y = ghd.ghd_linear(ctx, to_dev(x), to_dev(w))
+    ghd.ghd_sync_status(ctx)
+    assert max_rel_err(y.cpu().numpy(), oracle.linear(x, w)) <= 2e-6
+
+
+def _attention_case(ghd, shape, n, L, parent, splits, seed=400):
+    Lmax = L + n + 3
+    ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
+    if splits:
+        ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPLITS, splits)
+    H, dh, dt = shape.n_heads, shape.d_head, shape.dtype
+    q = wl.normal((n, H, dh), seed, dtype=dt)
+    kc = wl.normal((H, Lmax, dh), seed + 1, dtype=dt)      # rows [L, L+n) play the appended new rows
+    vc = wl.normal((H, Lmax, dh), seed + 2, dtype=dt)
+    vis, _, _ = oracle.tree_build(parent, L)
+    k_new = kc[:, L:L + n].transpose(1, 0, 2)
+    v_new = vc[:, L:L + n].transpose(1, 0, 2)
+    want = oracle.tree_attention(q, k_new, v_new, kc, vc, L, vis)
+    tree = ghd.ghd_tree_build(ctx, parent, L)
+    out = ghd.ghd_tree_attention(ctx, to_dev(q.reshape(n, H * dh)), ghd.KvLayer(to_dev(kc), to_dev(vc), L), tree)
+    ghd.ghd_sync_status(ctx)
+    return max_rel_err(out.cpu().numpy().reshape(n, H, dh), want)
+
+
+ATTN_CASES = [(1, 0, 0), (1, 1, 1), (8, 256, 0), (9, 63, 1), (33, 65, 3), (64, 300, 0), (64, 300, 16), (130, 17, 2),
+              (256, 129, 0)]
+
+
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
+@pytest.mark.parametrize("n,L,splits", ATTN_CASES)
+def test_tree_attention(ghd, shape, n, L, splits):
+    parent = wl.random_tree(n, 8, 1000 + n, max_children=6)
+    err = _attention_case(ghd, shape, n, L, parent, splits)
+    assert err <= (2e-5 if shape.dtype == "f32" else 2e-3)
+
+
+def test_chain_tree_is_causal_attention_and_star_sees_only_root(ghd):
+    for parent in (wl.chain_tree(40), wl.star_tree(40)):
+        assert _attention_case(ghd, SMALL32, 40, 50, parent, 0) <= 2e-5
+
+
+def test_argmax_bit_exact_including_ties(ghd):
+    ctx = make_ctx(ghd, SMALL32, 128, 64)
+    v = 32000
+    lg = wl.normal((9, v), 500).astype(np.float32)
+    lg[1, 100] = lg[1, 31999] = 50.0            # tie -> first index
+    lg[2, :] = 0.0                              # all equal -> 0
+    lg[3, 31999] = 60.0                         # maximum in the last column
+    lg[4, 0] = 60.0
+    lg[5, 777] = lg[5, 778] = 55.0
+    out = ghd.ghd_argmax(ctx, to_dev(lg))
+    ghd.ghd_sync_status(ctx)
+    assert np.array_equal(out.cpu().numpy(), oracle.argmax(lg))
+    small = wl.normal((3, 5), 501).astype(np.float32)
+    assert np.array_equal(ghd.ghd_argmax(ctx, to_dev(small)).cpu().numpy(), oracle.argmax(small))
+
+
+def _accept_gpu(ghd, ctx, parent, tokens, amax):
+    tree = ghd.ghd_tree_build(ctx, parent, 0)
+    res = ghd.ghd_accept(ctx, tree, to_dev(np.asarray(tokens, np.int32)), to_dev(np.asarray(amax, np.int32)))
+    r = res.cpu().numpy()
+    m = int(r[0])
+    return m, int(r[1]), r[2:2 + m + 1], r[2 + 256:2 + 256 + m + 1]
+
+
+def test_accept_bit_exact(ghd):
+    ctx = make_ctx(ghd, SMALL32, 1024, 256)
+    cases = []
+    for n in (1, 2, 3, 4):                                   # all small trees, binary alphabet (duplicates included)
+        for rest in itertools.product(*[range(i) for i in range(1, n)]):
+            for bits in itertools.product((0, 1), repeat=2 * n):
+                cases.append(([-1] + list(rest), bits[:n], bits[n:]))
+    rng = wl.Rng(77)
+    for trial in range(40):                                  # bigger trees with planted partial matches
+        n = [5, 17, 64, 65, 200, 256][trial % 6]
+        parent = wl.random_tree(n, 8, 600 + trial, max_children=6)
+        tokens = wl.draft_tokens(parent, 50, 700 + trial)
+        amax = np.array([rng.below(50) for _ in range(n)], dtype=np.int32)
+        for c in range(1, n):
+            if rng.below(3):
+                amax[parent[c]] = tokens[c]
+        cases.append((parent, tokens, amax))
+    for parent, tokens, amax in cases:
+        m, emitted, nodes, toks = _accept_gpu(ghd, ctx, parent, tokens, amax)
+        wm, wnodes, wtoks = oracle.accept(parent, tokens, amax)
+        assert (m, emitted) == (wm, wm + 1)
+        assert np.array_equal(nodes, wnodes) and np.array_equal(toks, wtoks)
+    ghd.ghd_sync_status(ctx)
+
+
+# ---------------------------------------------------------------- layer
+def _layer_case(ghd, shape, config_id, n, L, parent, vis=None, depth=None, gains=True, opts=()):
+    Lmax = L + n
+    ctx = make_ctx(ghd, shape, Lmax, max(n, 1))
+    for o, v in opts:
+        ghd.ghd_set_option(ctx, o, v)
+    w = wl.layer_weights(shape, config_id, 0, random_gains=gains)
+    kc, vc = wl.kv_cache(shape, config_id, 0, L, Lmax)
+    x = wl.layer_input(shape, config_id, n)
+    if vis is None:
+        ovis, _, opos = oracle.tree_build(parent, L)
+        tree = ghd.ghd_tree_build(ctx, parent, L)
+    else:
+        ovis, opos = vis.astype(np.uint8), (L + depth).astype(np.int32)
+        tree = ghd.ghd_tree_from_mask(ctx, ghd.pack_mask(vis), L, depth=depth)
+    okc, ovc = kc.copy(), vc.copy()
+    want = oracle.layer(shape, w, okc, ovc, L, ovis, opos, x)
+    kv = ghd.KvLayer(to_dev(kc), to_dev(vc), L)
+    y = ghd.ghd_verify_layer(ctx, gpu_layer_weights(w), kv, tree, to_dev(x))
+    ghd.ghd_sync_status(ctx)
+    tol = tol_for(shape.dtype)
+    assert max_rel_err(y.float().cpu().numpy(), want) <= tol
+    gk, gv = kv.k.float().cpu().numpy(), kv.v.float().cpu().numpy()
+    assert np.array_equal(gk[:, :L], kc[:, :L].astype(np.float32))       # old rows untouched
+    assert max_rel_err(gk[:, L:], okc[:, L:]) <= tol and max_rel_err(gv[:, L:], ovc[:, L:]) <= tol
+    return ctx
+
+
+def test_config1_tiny_layer_f32(ghd):
+    """d_model 512, 8 heads x 64, FFN 1376, KV 256, 8-node random tree of depth <= 4."""
+    _layer_case(ghd, wl.TINY, 1, 8, 256, wl.random_tree(8, 4, wl.BASE_SEED + 1000))
+
+
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
+@pytest.mark.parametrize("n,L", [(1, 0), (1, 40), (13, 100), (64, 77), (100, 300)])
+def test_small_layers(ghd, shape, n, L):
+    _layer_case(ghd, shape, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6))
+
+
+def test_config2_llama7b_layer_f16(ghd):
+    """LLaMA-7B-shaped layer, half weights, KV 1024, 64-node Medusa-style tree."""
+    _layer_case(ghd, wl.LLAMA7B, 2, 64, 1024, wl.medusa_tree(64), gains=False)
+
+
+def test_layer_with_explicit_lookahead_mask(ghd):
+    vis, depth, parent = wl.lookahead_pattern(7, 5, 5)
+    _layer_case(ghd, SMALL16_DH128, 12, len(parent), 200, parent, vis=vis, depth=depth)
+
+
+# ---------------------------------------------------------------- step
+def _model(ghd, shape, config_id, L, Lmax):
+    head = wl.head_weights(shape, config_id)
+    layers = [wl.layer_weights(shape, config_id, l, random_gains=True) for l in range(shape.n_layers)]
+    caches = [wl.kv_cache(shape, config_id, l, L, Lmax) for l in range(shape.n_layers)]
+    gw = ghd.ModelWeights(to_dev(head["embed"]), [gpu_layer_weights(w) for w in layers], to_dev(head["rms_final"]),
+                          to_dev(head["lm_head"]))
+    gkv = [ghd.KvLayer(to_dev(k), to_dev(v), L) for k, v in caches]
+    return head, layers, caches, gw, gkv
+
+
+@pytest.mark.parametrize("shape,graph", [(SMALL32, 0), (SMALL16, 0), (SMALL16, 2)], ids=["f32", "f16", "f16graph"])
+def test_small_step_logits_argmax_accept(ghd, shape, graph):
+    n, L = 24, 90
+    Lmax = L + n
+    parent = wl.random_tree(n, 6, 801, max_children=4)
+    tokens = wl.draft_tokens(parent, shape.vocab, 802)
+    head, layers, caches, gw, gkv = _model(ghd, shape, 13, L, Lmax)
+    vis, _, pos = oracle.tree_build(parent, L)
+    want_logits, want_amax = oracle.step(shape, head, layers, caches, L, vis, pos, tokens)
+    # plant a two-token accepted path so that acceptance is not trivially zero
+    c1 = parent.index(0)
+    tokens[c1] = want_amax[0]
+    want_logits, want_amax = oracle.step(shape, head, layers, [wl.kv_cache(shape, 13, l, L, Lmax) for l in range(shape.n_layers)],
+                                         L, vis, pos, tokens)
+    ctx = make_ctx(ghd, shape, Lmax, n)
+    ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, graph)
+    tree = ghd.ghd_tree_build(ctx, parent, L)
+    tok_d = to_dev(tokens)
+    for _ in range(2 if graph else 1):                        # second call replays the captured graph
+        logits, amax = ghd.ghd_verify_step(ctx, gw, gkv, tree, tok_d)
+    res = ghd.ghd_accept(ctx, tree, tok_d, amax).cpu().numpy()
+    ghd.ghd_sync_status(ctx)
+    got = logits.cpu().numpy()
+    assert max_rel_err(got, want_logits) <= tol_for(shape.dtype)
+    assert argmax_margin_ok(want_logits, np.abs(got - want_logits).max()), "seed gives a near-tie; pick another"
+    assert np.array_equal(amax.cpu().numpy(), want_amax)
+    m, nodes, toks = oracle.accept(parent, tokens, want_amax)
+    assert m >= 1 and res[0] == m and res[1] == m + 1
+    assert np.array_equal(res[2:3 + m], nodes) and np.array_equal(res[258:259 + m], toks)
+
+
+def test_width1_chain_reproduces_sequential_greedy_steps_on_gpu(ghd):
+    shape, k, L = SMALL32, 5, 30
+    Lmax = L + k + 1
+    head, layers, _, gw, _ = _model(ghd, shape, 14, L, Lmax)
+    ctx = make_ctx(ghd, shape, Lmax, k + 1)
+    fresh = lambda: [ghd.KvLayer(to_dev(kc), to_dev(vc), L) for kc, vc in
+                     (wl.kv_cache(shape, 14, l, L, Lmax) for l in range(shape.n_layers))]
+    gkv = fresh()
+    tok, seq = 5, []
+    for s in range(k + 1):                                    # sequential decoding, one node per step
+        for kv in gkv:
+            kv.len = L + s
+        tree = ghd.ghd_tree_build(ctx, [-1], L + s)
+        _, am = ghd.ghd_verify_step(ctx, gw, gkv, tree, to_dev(np.array([tok], np.int32)))
+        tok = int(am.cpu()[0])
+        seq.append(tok)
+    parent = wl.chain_tree(k + 1)
+    tree = ghd.ghd_tree_build(ctx, parent, L)
+    tokens = to_dev(np.array([5] + seq[:k], np.int32))
+    _, am = ghd.ghd_verify_step(ctx, gw, fresh(), tree, tokens)
+    res = ghd.ghd_accept(ctx, tree, tokens, am).cpu().numpy()
+    ghd.ghd_sync_status(ctx)
+    assert list(am.cpu().numpy()) == seq
+    assert res[0] == k and list(res[258:259 + k]) == seq
