@@ -144,7 +144,7 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
     chunk = ((chunk + TK - 1) / TK) * TK;
     dim3 grid((t->n + QB - 1) / QB, m.n_heads, splits);
 #define GHD_ATTN(T, DH)                                                                                          \
-    k_attn_simt<T, DH><<<grid, QB * 32, 0, c->stream>>>((const T*)q, (const T*)kv->k, (const T*)kv->v, t->mask,  \
+    k_attn_simt<T, DH><<<grid, QB * 32, 0, c->cur>>>((const T*)q, (const T*)kv->k, (const T*)kv->v, t->mask,  \
                                                         t->n_words, t->n, m.n_heads, t->kv_len, m.max_kv_len,    \
                                                         chunk, c->att_o, c->att_ml, m.max_nodes)
     if (m.dtype == GHD_F32) { if (m.d_head == 64) GHD_ATTN(float, 64); else GHD_ATTN(float, 128); }
@@ -153,10 +153,10 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
     c->launches++;
     dim3 cgrid(t->n, m.n_heads);
     if (m.dtype == GHD_F32)
-        k_attn_combine<float><<<cgrid, m.d_head, 0, c->stream>>>(c->att_o, c->att_ml, (float*)out, splits, m.n_heads,
+        k_attn_combine<float><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (float*)out, splits, m.n_heads,
                                                                  m.d_head, m.max_nodes);
     else
-        k_attn_combine<__half><<<cgrid, m.d_head, 0, c->stream>>>(c->att_o, c->att_ml, (__half*)out, splits, m.n_heads,
+        k_attn_combine<__half><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (__half*)out, splits, m.n_heads,
                                                                   m.d_head, m.max_nodes);
     c->launches++;
 }

@@ -81,9 +81,9 @@ k_gemm_simt(const T* __restrict__ x, const T* __restrict__ w, float* __restrict_
 void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, float* y) {
     dim3 grid((m + WARPS - 1) / WARPS, (n + NG - 1) / NG);
     if (c->cfg.dtype == GHD_F32)
-        k_gemm_simt<float><<<grid, WARPS * 32, 0, c->stream>>>((const float*)x, (const float*)w, y, n, k, m);
+        k_gemm_simt<float><<<grid, WARPS * 32, 0, c->cur>>>((const float*)x, (const float*)w, y, n, k, m);
     else
-        k_gemm_simt<__half><<<grid, WARPS * 32, 0, c->stream>>>((const __half*)x, (const __half*)w, y, n, k, m);
+        k_gemm_simt<__half><<<grid, WARPS * 32, 0, c->cur>>>((const __half*)x, (const __half*)w, y, n, k, m);
     c->launches++;
 }
 

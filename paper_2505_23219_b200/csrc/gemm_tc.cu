@@ -1,6 +1,547 @@
-// placeholder until the tcgen05 kernel lands
+// Skinny projection GEMM on the 5th-generation tensor cores (sm_100a), half in,
+// float accumulate:  Y[n][m] = X[n][k] * W[m][k]^T  with n <= 256 tree nodes.
+//
+// The problem is transposed for the hardware ("swap A/B"): a tile is 128 output
+// features (rows of W, the MMA M dimension) by all NB = roundup16(n) nodes (the
+// MMA N dimension), so each weight byte is fetched from HBM exactly once and the
+// node columns stay on-chip.  The accumulator tile [128 x NB] float lives in
+// tensor memory (TMEM), double-buffered so that the epilogue of one tile overlaps
+// the MMAs of the next.
+//
+// Work split (stream-K): the (tile, 64-wide k-step) iteration space is flattened
+// and cut into equal contiguous ranges, one per CTA (one CTA per SM), so every SM
+// streams the same number of weight bytes whatever the tile count.  A CTA whose
+// range covers only part of a tile's k-steps writes its float partial tile to the
+// workspace and bumps the tile's arrival counter; whichever CTA arrives last sums
+// the partials in CTA order (fixed order -> bit-reproducible) and runs the
+// epilogue.  Nobody ever waits for another CTA.
+//
+// Per CTA: warp 0 = TMA producer (weights and activations into a ring of
+// 128B-swizzled shared-memory stages), warp 1 = MMA issuer (tcgen05.mma, one
+// thread) and TMEM owner, warps 2..5 = epilogue (tcgen05.ld, fused epilogue).
+// All mbarrier waits are bounded: on expiry the kernel records a status code,
+// stops issuing work, drains what it issued, frees its TMEM and returns.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstring>
+
 #include "internal.h"
+
 namespace ghd {
-bool gemm_tc_supported(const ghd_ctx*, int, int, int, int) { return false; }
-ghd_status launch_gemm_tc(ghd_ctx*, const void*, const void*, int, int, int, const EpiArgs&) { return GHD_EUNSUPPORTED; }
+
+namespace {
+
+constexpr int TILE_M = 128;          // output features per tile (MMA M)
+constexpr int TILE_K = 64;           // halfs per k-step = one 128-byte swizzle row
+constexpr int UMMA_K = 16;           // k per tcgen05.mma of kind::f16
+constexpr int MAX_STAGES = 10;
+constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
+constexpr int THREADS = 192;
+constexpr uint32_t SPIN_LIMIT = 1u << 22;
+
+struct GemmParams {
+    int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
+    int n_tiles, kiters, stages;
+    int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
+    float* part;                     // [ctas][2][nb][128] float partial tiles
+    int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
+    int* status;
+    EpiArgs epi;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (after recording `code`) when the phase never completes
+// or another role of this CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+    for (uint32_t spin = 0; spin < SPIN_LIMIT; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if (spin > 64) {
+            if (*abort_flag) return false;
+            __nanosleep(spin > 4096 ? 256 : 32);
+        }
+    }
+    *abort_flag = 1;
+    atomicCAS(status, DEV_OK, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 lanes x 32 consecutive columns of 32-bit accumulators -> 32 registers per thread.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 64
+// halfs (128 B), 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor of kind::f16: half A and B (both K-major), float D, M = 128, N = nb.
+__device__ __forceinline__ uint32_t instr_desc_f16(int nb) {
+    return (1u << 4) | ((uint32_t)(nb >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+}
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// First CTA whose iteration range contains flattened iteration `it` (ranges are
+// [total*c/G, total*(c+1)/G) and G <= total, so none is empty).
+__device__ __forceinline__ int cta_of_iter(long long it, long long total, int G) {
+    return (int)(((it + 1) * G + total - 1) / total) - 1;
+}
+
+struct Smem {
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int last_flag;
+    float stage_x[EPI_CHUNK][TILE_M + 1];   // epilogue exchange buffer (rotary pairs, gate/up pairs)
+};
+
+// ---------------------------------------------------------------- fused epilogue
+// Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature
+// for nodes c0 .. c0+31.
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, int tile, int row, int c0, float (&v)[32]) {
+    const EpiArgs& e = p.epi;
+    if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
+        const int f = tile * TILE_M + row;
+        if (f < p.m) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int node = c0 + j;
+                if (node < p.n) {
+                    float* dst = e.out_f32 + (size_t)node * p.m + f;
+                    *dst = (e.mode == EPI_RESID) ? (*dst + v[j]) : v[j];
+                }
+            }
+        }
+        return;
+    }
+    if (e.mode == EPI_SWIGLU) {
+        // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
+        epi_bar();
+        if (row < 64) {
+            const int f = tile * 64 + row;
+            __half* u = (__half*)e.out_t;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int node = c0 + j;
+                if (node < p.n) {
+                    const float g = v[j], up = sm->stage_x[j][row + 64];
+                    u[(size_t)node * p.swiglu_f + f] = __float2half_rn(g / (1.f + __expf(-g)) * up);
+                }
+            }
+        }
+        epi_bar();
+        return;
+    }
+    // EPI_ROPE_KV: output features [0,d) = q, [d,2d) = k, [2d,3d) = v; tiles never straddle sections
+    const int d = e.d_model, dh = e.d_head, half = dh >> 1;
+    const int f = tile * TILE_M + row;
+    const int section = f / d, el = f - section * d;
+    const int head = el / dh, idx = el - head * dh;
+    if (section < 2) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
+        epi_bar();
+        const int prow = (idx < half) ? row + half : row - half;
+        const int t = (idx < half) ? idx : idx - half;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const int node = c0 + j;
+            if (node < p.n) {
+                const float2 cs = *reinterpret_cast<const float2*>(e.rope + (size_t)node * dh + 2 * t);
+                const float other = sm->stage_x[j][prow];
+                const float r = (idx < half) ? (v[j] * cs.x - other * cs.y) : (v[j] * cs.x + other * cs.y);
+                if (section == 0)
+                    ((__half*)e.out_t)[(size_t)node * d + el] = __float2half_rn(r);
+                else
+                    ((__half*)e.k_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(r);
+            }
+        }
+        epi_bar();
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const int node = c0 + j;
+            if (node < p.n)
+                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(v[j]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* tiles = smem_raw + pad;
+    const uint32_t a_bytes = TILE_M * TILE_K * 2, b_bytes = (uint32_t)p.nb * TILE_K * 2;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+    Smem* sm = reinterpret_cast<Smem*>(tiles + (size_t)p.stages * stage_bytes);
+    const uint32_t tiles_addr = smem_u32(tiles);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const long long total = (long long)p.n_tiles * p.kiters;
+    const long long it_beg = total * cta / G, it_end = total * (cta + 1) / G;
+
+    // accumulator buffers are EPI_CHUNK-aligned so that a 32-column read never leaves the allocation
+    const uint32_t buf_cols = (uint32_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK);
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * buf_cols) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&sm->full[s]), 1); mbar_init(smem_u32(&sm->empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), 4); }
+        mbar_init(smem_u32(&sm->drain), 1);
+        sm->abort_flag = 0;
+        sm->last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint64_t pol_stream, pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            uint32_t stage = 0, phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (long long it = it_beg; it < it_end && ok; ++it) {
+                const int tile = (int)(it / p.kiters), kk = (int)(it - (long long)tile * p.kiters);
+                if (issued >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+                if (!ok) break;
+                const uint32_t full = smem_u32(&sm->full[stage]);
+                const uint32_t a_dst = tiles_addr + stage * stage_bytes, b_dst = a_dst + a_bytes;
+                mbar_expect_tx(full, stage_bytes);
+                if (p.swiglu_f) {
+                    tma_load_2d(a_dst, &tm_w, kk * TILE_K, tile * 64, full, pol_stream);
+                    tma_load_2d(a_dst + a_bytes / 2, &tm_w, kk * TILE_K, p.swiglu_f + tile * 64, full, pol_stream);
+                } else {
+                    tma_load_2d(a_dst, &tm_w, kk * TILE_K, tile * TILE_M, full, pol_stream);
+                }
+                tma_load_2d(b_dst, &tm_x, kk * TILE_K, 0, full, pol_keep);
+                ++issued;
+                if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) {
+                // drain: wait (bounded) until every load issued into the ring has landed
+                const long long inflight = issued < p.stages ? issued : p.stages;
+                uint32_t s = stage, ph = phase;
+                for (long long q = 0; q < inflight; ++q) {
+                    if (s == 0) { s = p.stages - 1; ph ^= 1; } else --s;
+                    for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->full[s]), ph); ++spin) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_f16(p.nb);
+            uint32_t stage = 0, phase = 0, buf = 0, buf_phase = 0;
+            long long units = 0;
+            bool ok = true;
+            long long it = it_beg;
+            while (it < it_end && ok) {
+                const int tile = (int)(it / p.kiters), k0 = (int)(it - (long long)tile * p.kiters);
+                const long long left = it_end - it;
+                const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
+                if (units >= 2) ok = mbar_wait(smem_u32(&sm->tmem_empty[buf]), buf_phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMEM);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * buf_cols;
+                for (int kk = k0; kk < k1; ++kk) {
+                    ok = mbar_wait(smem_u32(&sm->full[stage]), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = tiles_addr + stage * stage_bytes, b_addr = a_addr + a_bytes;
+                    const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(b_addr);
+#pragma unroll
+                    for (int j = 0; j < TILE_K / UMMA_K; ++j)   // +32 bytes along k inside the swizzle row per step
+                        tc_mma_f16(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, (kk > k0 || j > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&sm->empty[stage]));    // stage is free once these MMAs have read it
+                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&sm->tmem_full[buf]));       // accumulator complete
+                ++units;
+                if (++buf == 2) { buf = 0; buf_phase ^= 1; }
+                it += (k1 - k0);
+            }
+            if (!ok) {
+                // make sure no MMA is still running before TMEM goes away
+                tc_commit(smem_u32(&sm->drain));
+                for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain), 0); ++spin) __nanosleep(64);
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue warps (TMEM lanes 32*(warp%4) ..)
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int et = threadIdx.x - 64;                       // 0..127 among epilogue threads
+        uint32_t buf = 0, buf_phase = 0;
+        bool ok = true;
+        long long it = it_beg;
+        const size_t slot_elems = (size_t)p.nb * TILE_M;
+        while (it < it_end && ok) {
+            const int tile = (int)(it / p.kiters), k0 = (int)(it - (long long)tile * p.kiters);
+            const long long left = it_end - it;
+            const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
+            const bool whole = (k0 == 0 && k1 == p.kiters);
+            mbar_wait(smem_u32(&sm->tmem_full[buf]), buf_phase, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            epi_bar();                                         // all 128 threads take the same decision
+            ok = (*abort_flag == 0);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
+            if (whole) {
+                for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
+                    float v[32];
+                    tc_ld32(t_addr + c0, v);                   // may run past nb, never past the buffer
+                    if (c0 < p.n) epilogue_chunk(p, sm, tile, row, c0, v);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+            } else {
+                // partial tile: slot 0 when this is the CTA's first unit (it starts mid-tile or is
+                // its only unit of this tile), slot 1 when it is the head part of the CTA's last tile
+                const int slot = (it == it_beg) ? 0 : 1;
+                float* mine = p.part + ((size_t)cta * 2 + slot) * slot_elems;
+                for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
+                    float v[32];
+                    tc_ld32(t_addr + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + j < p.nb) mine[(size_t)(c0 + j) * TILE_M + row] = v[j];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+                __threadfence();
+                epi_bar();
+                const long long t_first = (long long)tile * p.kiters;
+                const int c_first = cta_of_iter(t_first, total, G), c_last = cta_of_iter(t_first + p.kiters - 1, total, G);
+                if (et == 0) {
+                    const int old = atomicAdd(p.counters + tile, 1);
+                    sm->last_flag = (old == c_last - c_first) ? 1 : 0;
+                }
+                epi_bar();
+                const bool last = sm->last_flag != 0;
+                epi_bar();
+                if (last) {
+                    __threadfence();
+                    for (int c0 = 0; c0 < p.nb && c0 < p.n; c0 += EPI_CHUNK) {
+                        float v[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        for (int c = c_first; c <= c_last; ++c) {
+                            const long long cb = total * c / G;
+                            const int cslot = (cb >= t_first) ? 0 : 1;
+                            const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (c0 + j < p.nb) v[j] += __ldcg(src + (size_t)(c0 + j) * TILE_M + row);
+                        }
+                        epilogue_chunk(p, sm, tile, row, c0, v);
+                    }
+                    if (et == 0) p.counters[tile] = 0;         // ready for the next launch
+                }
+            }
+            if (++buf == 2) { buf = 0; buf_phase ^= 1; }
+            it += (k1 - k0);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Row-major half matrix [rows][cols] -> tensor map with a (box_rows x 64) box, 128-byte swizzle, zero fill.
+bool get_tmap(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+    TmapKey key{ptr, rows, cols, box_rows, (uint32_t)TILE_K};
+    auto it = c->tmaps->find(key);
+    if (it != c->tmaps->end()) { memcpy(out, it->second.data(), sizeof(CUtensorMap)); return true; }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)TILE_K, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUtensorMap tm;
+    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::vector<uint64_t> blob(sizeof(CUtensorMap) / 8);
+    memcpy(blob.data(), &tm, sizeof(CUtensorMap));
+    if (c->tmaps->size() > 4096) c->tmaps->clear();
+    (*c->tmaps)[key] = blob;
+    *out = tm;
+    return true;
+}
+
+size_t smem_bytes_for(int nb, int stages) {
+    return 1024 + (size_t)stages * (TILE_M * TILE_K * 2 + (size_t)nb * TILE_K * 2) + sizeof(Smem);
+}
+
+int pick_stages(int nb) {
+    int s = MAX_STAGES;
+    while (s > 2 && smem_bytes_for(nb, s) > 227 * 1024) --s;
+    return s;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
+    if (c->cfg.dtype != GHD_F16 || n < 1 || n > GHD_MAX_NODES || k % 8 || k < TILE_K) return false;
+    const int n_tiles = (epi_mode == EPI_SWIGLU) ? (m / 2) / 64 : (m + TILE_M - 1) / TILE_M;
+    if (n_tiles < 1 || n_tiles > 4096) return false;
+    if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
+    if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
+    return true;
+}
+
+ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi) {
+    if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) {
+        snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: operands must be 16-byte aligned");
+        return GHD_EINVAL;
+    }
+    GemmParams p{};
+    p.n = n;
+    p.nb = ((n + 15) / 16) * 16;
+    p.k = k;
+    p.m = m;
+    p.swiglu_f = (epi.mode == EPI_SWIGLU) ? m / 2 : 0;
+    p.n_tiles = p.swiglu_f ? p.swiglu_f / 64 : (m + TILE_M - 1) / TILE_M;
+    p.kiters = (k + TILE_K - 1) / TILE_K;
+    p.stages = pick_stages(p.nb);
+    p.part = c->gemm_part;
+    p.counters = c->counters;
+    p.status = c->status;
+    p.epi = epi;
+    CUtensorMap tm_w, tm_x;
+    if (!get_tmap(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 64 : TILE_M, &tm_w) ||
+        !get_tmap(c, x, (uint64_t)n, (uint64_t)k, (uint32_t)p.nb, &tm_x)) {
+        snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: tensor map encoding failed");
+        return GHD_ECUDA;
+    }
+    const long long total = (long long)p.n_tiles * p.kiters;
+    int ctas = c->opt_gemm_ctas > 0 ? c->opt_gemm_ctas : c->sm_count;
+    if (ctas > c->sm_count) ctas = c->sm_count;
+    if (ctas > total) ctas = (int)total;
+    const size_t smem = smem_bytes_for(p.nb, p.stages);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+            snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
+            return GHD_ECUDA;
+        }
+        attr_set = true;
+    }
+    k_gemm_tc<<<ctas, THREADS, smem, c->cur>>>(tm_w, tm_x, p);
+    c->launches++;
+    return GHD_OK;
+}
+
+}  // namespace ghd

@@ -139,6 +139,8 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     memset(c->err, 0, sizeof(c->err));
     c->cfg = *cfg;
     c->stream = (cudaStream_t)cuda_stream;
+    c->cur = c->stream;
+    c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
     c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = 0;
@@ -156,6 +158,7 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
 void ghd_destroy(ghd_ctx* c) {
     if (!c) return;
     for (StepGraph* g : *c->graphs) { cudaGraphExecDestroy(g->exec); delete g; }
+    if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     delete c->graphs;
     delete c->tmaps;
     delete c;
@@ -292,11 +295,18 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
             c->launches += g->kernels;
             return GHD_OK;
         }
+    // The caller's stream may be the legacy default stream, which cannot be captured:
+    // record the kernels on a stream of our own (nothing executes there) and replay
+    // the instantiated graph on the caller's stream.
     const int64_t before = c->launches;
-    if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return check_cuda(c, "begin capture");
+    if (!c->cap_stream && cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess)
+        return check_cuda(c, "capture stream");
+    if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return check_cuda(c, "begin capture");
+    c->cur = c->cap_stream;
     s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev);
+    c->cur = c->stream;
     cudaGraph_t graph = nullptr;
-    const cudaError_t ce = cudaStreamEndCapture(c->stream, &graph);
+    const cudaError_t ce = cudaStreamEndCapture(c->cap_stream, &graph);
     if (s != GHD_OK) { if (graph) cudaGraphDestroy(graph); c->launches = before; return s; }
     if (ce != cudaSuccess || !graph) { c->launches = before; cudaGetLastError(); return fail(c, GHD_ECUDA, "stream capture failed"); }
     cudaGraphExec_t exec = nullptr;
@@ -359,7 +369,7 @@ ghd_status ghd_sync_status(ghd_ctx* c) {
     if (cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return check_cuda(c, "status read");
     if (st != DEV_OK) {
         snprintf(c->err, sizeof(c->err), "device wait expired (code %d)", st);
-        cudaMemset(c->status, 0, sizeof(int));
+        cudaMemset(c->status, 0, 256 + sizeof(int) * 4096);   // status word and tile arrival counters
         return GHD_ETIMEOUT;
     }
     return GHD_OK;

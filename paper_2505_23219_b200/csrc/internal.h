@@ -47,7 +47,9 @@ struct StepGraph;
 
 struct ghd_ctx {
     ghd_model_cfg cfg;
-    cudaStream_t stream;
+    cudaStream_t stream;      // the caller's stream
+    cudaStream_t cur;         // where launches go: `stream`, or `cap_stream` while a graph is being captured
+    cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
     int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas;

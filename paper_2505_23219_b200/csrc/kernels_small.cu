@@ -74,14 +74,14 @@ __global__ void k_tree_from_mask(int n, int n_words, int kv_len, int d_head, dou
 void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t) {
     ParentArg pa;
     for (int i = 0; i < GHD_MAX_NODES; ++i) pa.p[i] = (int16_t)(i < t->n ? parent_host[i] : -1);
-    k_tree_build<<<1, GHD_MAX_NODES, 0, c->stream>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
+    k_tree_build<<<1, GHD_MAX_NODES, 0, c->cur>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                      (double)c->cfg.rope_theta, t->mask, t->parent, t->depth,
                                                      t->pos, t->rope);
     c->launches++;
 }
 
 void launch_tree_from_mask(ghd_ctx* c, const ghd_tree* t, bool have_depth) {
-    k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->stream>>>(t->n, t->n_words, t->kv_len, c->cfg.d_head,
+    k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->cur>>>(t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                          (double)c->cfg.rope_theta, have_depth ? 1 : 0, t->mask,
                                                          t->depth, t->pos, t->rope);
     c->launches++;
@@ -114,22 +114,22 @@ static int grid_for(size_t count, int block, int cap) {
 void launch_load_x(ghd_ctx* c, const void* x_in, int n) {
     const size_t count = (size_t)n * c->cfg.d_model;
     const int g = grid_for(count, 256, 4 * c->sm_count);
-    GHD_DISPATCH_T(c, (k_load_x<float><<<g, 256, 0, c->stream>>>((const float*)x_in, c->xres, count)),
-                   (k_load_x<__half><<<g, 256, 0, c->stream>>>((const __half*)x_in, c->xres, count)));
+    GHD_DISPATCH_T(c, (k_load_x<float><<<g, 256, 0, c->cur>>>((const float*)x_in, c->xres, count)),
+                   (k_load_x<__half><<<g, 256, 0, c->cur>>>((const __half*)x_in, c->xres, count)));
     c->launches++;
 }
 
 void launch_store_x(ghd_ctx* c, void* x_out, int n) {
     const size_t count = (size_t)n * c->cfg.d_model;
     const int g = grid_for(count, 256, 4 * c->sm_count);
-    GHD_DISPATCH_T(c, (k_store_x<float><<<g, 256, 0, c->stream>>>(c->xres, (float*)x_out, count)),
-                   (k_store_x<__half><<<g, 256, 0, c->stream>>>(c->xres, (__half*)x_out, count)));
+    GHD_DISPATCH_T(c, (k_store_x<float><<<g, 256, 0, c->cur>>>(c->xres, (float*)x_out, count)),
+                   (k_store_x<__half><<<g, 256, 0, c->cur>>>(c->xres, (__half*)x_out, count)));
     c->launches++;
 }
 
 void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n) {
-    GHD_DISPATCH_T(c, (k_embed<float><<<n, 256, 0, c->stream>>>((const float*)embed, tokens, c->xres, c->cfg.d_model)),
-                   (k_embed<__half><<<n, 256, 0, c->stream>>>((const __half*)embed, tokens, c->xres, c->cfg.d_model)));
+    GHD_DISPATCH_T(c, (k_embed<float><<<n, 256, 0, c->cur>>>((const float*)embed, tokens, c->xres, c->cfg.d_model)),
+                   (k_embed<__half><<<n, 256, 0, c->cur>>>((const __half*)embed, tokens, c->xres, c->cfg.d_model)));
     c->launches++;
 }
 
@@ -166,8 +166,8 @@ __global__ void k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, 
 
 void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out) {
     const int d = c->cfg.d_model;
-    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, 256, 0, c->stream>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
-                   (k_rmsnorm<__half><<<n, 256, 0, c->stream>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
+    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, 256, 0, c->cur>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
+                   (k_rmsnorm<__half><<<n, 256, 0, c->cur>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
     c->launches++;
 }
 
@@ -201,9 +201,9 @@ void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, con
     const size_t total = (size_t)t->n * m.n_heads * (m.d_head / 2);
     const int g = grid_for(total, 256, 8 * c->sm_count);
     GHD_DISPATCH_T(c,
-        (k_rope_append<float><<<g, 256, 0, c->stream>>>(qkv_raw, t->rope, (float*)c->qbuf, (float*)kv->k, (float*)kv->v,
+        (k_rope_append<float><<<g, 256, 0, c->cur>>>(qkv_raw, t->rope, (float*)c->qbuf, (float*)kv->k, (float*)kv->v,
                                                          t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)),
-        (k_rope_append<__half><<<g, 256, 0, c->stream>>>(qkv_raw, t->rope, (__half*)c->qbuf, (__half*)kv->k, (__half*)kv->v,
+        (k_rope_append<__half><<<g, 256, 0, c->cur>>>(qkv_raw, t->rope, (__half*)c->qbuf, (__half*)kv->k, (__half*)kv->v,
                                                           t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)));
     c->launches++;
 }
@@ -222,8 +222,8 @@ __global__ void k_swiglu(const float* __restrict__ gu, T* __restrict__ u, int n,
 void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n) {
     const size_t total = (size_t)n * c->cfg.d_ffn;
     const int g = grid_for(total, 256, 8 * c->sm_count);
-    GHD_DISPATCH_T(c, (k_swiglu<float><<<g, 256, 0, c->stream>>>(gu_raw, (float*)c->ubuf, n, c->cfg.d_ffn)),
-                   (k_swiglu<__half><<<g, 256, 0, c->stream>>>(gu_raw, (__half*)c->ubuf, n, c->cfg.d_ffn)));
+    GHD_DISPATCH_T(c, (k_swiglu<float><<<g, 256, 0, c->cur>>>(gu_raw, (float*)c->ubuf, n, c->cfg.d_ffn)),
+                   (k_swiglu<__half><<<g, 256, 0, c->cur>>>(gu_raw, (__half*)c->ubuf, n, c->cfg.d_ffn)));
     c->launches++;
 }
 
@@ -234,7 +234,7 @@ __global__ void k_residual(float* __restrict__ xres, const float* __restrict__ p
 
 void launch_residual(ghd_ctx* c, const float* proj_raw, int n) {
     const size_t count = (size_t)n * c->cfg.d_model;
-    k_residual<<<grid_for(count, 256, 8 * c->sm_count), 256, 0, c->stream>>>(c->xres, proj_raw, count);
+    k_residual<<<grid_for(count, 256, 8 * c->sm_count), 256, 0, c->cur>>>(c->xres, proj_raw, count);
     c->launches++;
 }
 
@@ -275,7 +275,7 @@ __global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __res
 }
 
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out) {
-    k_argmax<<<n, 512, 0, c->stream>>>(logits, v, out);
+    k_argmax<<<n, 512, 0, c->cur>>>(logits, v, out);
     c->launches++;
 }
 
@@ -319,7 +319,7 @@ __global__ void k_accept(int n, const int32_t* __restrict__ parent,
 }
 
 void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out) {
-    k_accept<<<1, GHD_MAX_NODES, 0, c->stream>>>(t->n, t->parent, tokens, amax, out);
+    k_accept<<<1, GHD_MAX_NODES, 0, c->cur>>>(t->n, t->parent, tokens, amax, out);
     c->launches++;
 }
 

@@ -129,6 +129,31 @@ def test_linear_cuda_core_path(ghd, shape, n, k, m):
     assert max_rel_err(y.cpu().numpy(), oracle.linear(x, w)) <= 2e-6
 
 
+TC_SHAPES = [(1, 64, 128), (5, 256, 40), (16, 512, 256), (17, 352, 130), (64, 4096, 1024), (64, 11008, 512),
+             (100, 1024, 1001), (128, 512, 384), (200, 2048, 256), (256, 1024, 640)]
+
+
+@pytest.mark.parametrize("n,k,m", TC_SHAPES)
+def test_linear_tcgen05_path(ghd, n, k, m):
+    ctx = make_ctx(ghd, SMALL16, 128, 256)
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PATH, 2)
+    x = wl.normal((n, k), 321, 1.0, dtype="f16")
+    w = wl.normal((m, k), 322, 0.02, dtype="f16")
+    xd, wd = to_dev(x), to_dev(w)
+    y = ghd.ghd_linear(ctx, xd, wd)
+    ghd.ghd_sync_status(ctx)
+    want = oracle.linear(x, w)
+    assert max_rel_err(y.cpu().numpy(), want) <= 2e-5        # exact products, float accumulation
+    y2 = ghd.ghd_linear(ctx, xd, wd)
+    ghd.ghd_sync_status(ctx)
+    assert np.array_equal(y.cpu().numpy(), y2.cpu().numpy())  # fixed reduction order -> reproducible
+    for ctas in (1, 7, 64):                                   # result must not depend on the work split
+        ghd.ghd_set_option(ctx, ghd.OPT_GEMM_CTAS, ctas)
+        y3 = ghd.ghd_linear(ctx, xd, wd)
+        ghd.ghd_sync_status(ctx)
+        assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
+
+
 def _attention_case(ghd, shape, n, L, parent, splits, seed=400):
     Lmax = L + n + 3
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
@@ -248,9 +273,23 @@ def test_config1_tiny_layer_f32(ghd):
 
 
 @pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
-@pytest.mark.parametrize("n,L", [(1, 0), (1, 40), (13, 100), (64, 77), (100, 300)])
+@pytest.mark.parametrize("n,L", [(1, 0), (1, 40), (13, 100), (64, 77), (100, 300), (256, 31)])
 def test_small_layers(ghd, shape, n, L):
     _layer_case(ghd, shape, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6))
+
+
+@pytest.mark.parametrize("n,L", [(1, 40), (13, 100), (64, 77)])
+def test_small_layers_half_on_cuda_cores(ghd, n, L):
+    import paper_2505_23219_b200 as g
+    _layer_case(ghd, SMALL16_DH128, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6),
+                opts=[(g.OPT_GEMM_PATH, 1), (g.OPT_ATTN_PATH, 1)])
+
+
+@pytest.mark.parametrize("n,L", [(1, 40), (13, 100), (64, 77), (200, 5)])
+def test_small_layers_forced_tcgen05_gemm(ghd, n, L):
+    import paper_2505_23219_b200 as g
+    _layer_case(ghd, SMALL16_DH128, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6),
+                opts=[(g.OPT_GEMM_PATH, 2)])
 
 
 def test_config2_llama7b_layer_f16(ghd):
