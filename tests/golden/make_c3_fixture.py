@@ -88,6 +88,7 @@ def main():
         "logits_abs_max": float(np.abs(logits).max()),
         "min_top2_margin": float(margins.min()),
         "row_margins": [float(f"{v:.6e}") for v in margins],
+        "runner_up": [int(np.argsort(logits[i])[-2]) for i in range(N)],
         "logit_samples": samples,
     }
     path = Path(__file__).resolve().parent / "c3_step_llama7b.json"
