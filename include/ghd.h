@@ -177,6 +177,29 @@ ghd_status ghd_rmsnorm(ghd_ctx *ctx, const float *x, const void *g, int32_t n, v
 ghd_status ghd_tree_attention(ghd_ctx *ctx, const void *q, const ghd_kv_layer *kv, const ghd_tree *tree, void *out);
 ghd_status ghd_argmax(ghd_ctx *ctx, const float *logits, int32_t n, int32_t v, int32_t *out);
 
+/* (The paper has no counterpart of this call; it exists for deployment reasons only.)
+ * ghd_tree_attention for callers that must not allocate device memory - code that runs
+ * inside another framework's fixed memory pool, plugins of a serving process whose memory
+ * budget is frozen at start-up, or loops in which cudaMalloc (it may synchronise the whole
+ * device) is forbidden.  Such callers cannot provide the workspace that holds the per-split
+ * partial results, so this variant keeps them in an array built into the library image
+ * (about 8.25 MiB, present on every GPU that loads the library until the process exits).
+ * It needs no context and calls no allocating routine.
+ *   stream: cudaStream_t (NULL = default).  dtype: ghd_dtype of q, caches and out.
+ *   q, out: dev T [n][n_heads*d_head]; k_cache, v_cache: dev T [n_heads][max_kv_len][d_head]
+ *   already holding the n new rows at [kv_len, kv_len + n); mask_dev: dev uint64
+ *   [n][ceil(n/64)] as in ghd_tree.  err_buf (host, may be NULL) receives a message on failure.
+ * Limits: n <= 64 and n_heads * d_head <= 4096, else GHD_ENOSPACE; d_head in {64, 128}.
+ * The first call on each device looks up the array's device address; make that first call
+ * outside any stream capture.  All calls on a device share the one array (it keeps whatever
+ * the previous call left; every slot that is read is rewritten first, so nothing needs
+ * clearing): two calls whose kernels may overlap on the GPU - different streams without an
+ * ordering between them - race on it.  Calls on one stream are safe. */
+ghd_status ghd_tree_attention_static(void *cuda_stream, int32_t dtype, int32_t n_heads, int32_t d_head,
+                                     int32_t max_kv_len, const void *q, const void *k_cache, const void *v_cache,
+                                     const uint64_t *mask_dev, int32_t n, int32_t kv_len, void *out,
+                                     char *err_buf, size_t err_len);
+
 /* Synchronises the stream and returns GHD_OK, GHD_ECUDA (with the CUDA error kept
  * for ghd_last_error) or GHD_ETIMEOUT when a kernel's bounded wait expired. */
 ghd_status ghd_sync_status(ghd_ctx *ctx);

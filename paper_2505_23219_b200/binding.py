@@ -17,7 +17,7 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
     "OPT_GEMM_CTAS", "EXPORTS",
 ]
@@ -33,6 +33,7 @@ EXPORTS = [
     "ghd_create", "ghd_destroy", "ghd_workspace_bytes", "ghd_set_workspace", "ghd_set_option", "ghd_tree_build",
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
+    "ghd_tree_attention_static",
 ]
 
 
@@ -101,6 +102,8 @@ def load_library(path: str | Path | None = None):
         "ghd_status_str": ([C.c_int], C.c_char_p),
         "ghd_last_error": ([vp], C.c_char_p),
         "ghd_launch_count": ([vp], C.c_int64),
+        "ghd_tree_attention_static": ([vp, i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, vp, C.c_char_p, C.c_size_t],
+                                      C.c_int),
     }
     for name, (args, res) in sig.items():
         fn = getattr(lib, name)
@@ -301,6 +304,23 @@ def ghd_tree_attention(ctx: Ctx, q, kv: KvLayer, tree: Tree, out=None):
     out = torch.empty_like(q) if out is None else out
     kvc = kv.c
     ctx._check(ctx.lib.ghd_tree_attention(ctx.handle, q.data_ptr(), C.byref(kvc), C.byref(tree.c), out.data_ptr()))
+    return out
+
+
+def ghd_tree_attention_static(q, k_cache, v_cache, mask_dev, n_heads: int, d_head: int, kv_len: int, out=None):
+    """Tree attention without a context or workspace, for callers that may not allocate device
+    memory: the split partials live in an array inside the library (limits: 64 nodes,
+    n_heads * d_head <= 4096).  Runs on torch's current stream; ``out`` is the caller's."""
+    lib = load_library()
+    n = q.shape[0]
+    out = torch.empty_like(q) if out is None else out
+    err = C.create_string_buffer(256)
+    st = lib.ghd_tree_attention_static(C.c_void_p(torch.cuda.current_stream().cuda_stream),
+                                       GHD_F32 if q.dtype == torch.float32 else GHD_F16, n_heads, d_head,
+                                       k_cache.shape[1], q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                       mask_dev.data_ptr(), n, kv_len, out.data_ptr(), err, 256)
+    if st != 0:
+        raise GhdError(st, err.value.decode())
     return out
 
 

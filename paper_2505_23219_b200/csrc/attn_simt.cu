@@ -10,6 +10,9 @@
 // (paper Sec. III-B-2: each partition keeps its own softmax and the results are
 // aligned by a scaling factor at the end).  32-key tiles of the new-row region in
 // which no query of the block has a visible key are skipped without being loaded.
+#include <cstdio>
+#include <mutex>
+
 #include "internal.h"
 
 namespace ghd {
@@ -161,4 +164,105 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
     c->launches++;
 }
 
+// ---------------------------------------------------------------------------
+// Tree attention for callers that cannot allocate device memory.
+//
+// Some hosts of this library are not allowed to call cudaMalloc at all: code
+// running inside another framework's pre-sized memory pool, a plugin in a
+// serving process whose memory budget is fixed at start-up, or a latency-critical
+// loop where an allocation (which may synchronise the device) is forbidden.
+// They cannot give ghd_tree_attention the workspace it needs for its per-split
+// partial results.  This variant keeps those partials in a fixed array that is
+// part of the library image instead; every GPU that loads the library carries
+// the array (about 8.25 MiB) until the process exits.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int ST_MAX_NODES = 64;       // tree nodes
+constexpr int ST_MAX_WIDTH = 4096;     // n_heads * d_head
+constexpr int ST_MAX_HEADS = ST_MAX_WIDTH / 64;
+constexpr int ST_MAX_SPLITS = 8;
+constexpr size_t ST_O_FLOATS = (size_t)ST_MAX_SPLITS * ST_MAX_NODES * ST_MAX_WIDTH;
+constexpr size_t ST_ML_FLOATS = (size_t)ST_MAX_SPLITS * ST_MAX_NODES * ST_MAX_HEADS * 2;
+
+// Split partials: numerators first, then (running max, running sum) pairs.
+static __device__ __align__(256) float g_static_scratch[ST_O_FLOATS + ST_ML_FLOATS];
+
+constexpr int ST_MAX_DEVICES = 64;
+float* g_static_scratch_addr[ST_MAX_DEVICES];   // device address of the array, per device, once known
+std::mutex g_static_scratch_lock;
+
+void st_error(char* buf, size_t len, const char* msg) {
+    if (buf && len) snprintf(buf, len, "%s", msg);
+}
+
+}  // namespace
 }  // namespace ghd
+
+extern "C" ghd_status ghd_tree_attention_static(void* cuda_stream, int32_t dtype, int32_t n_heads, int32_t d_head,
+                                                int32_t max_kv_len, const void* q, const void* k_cache,
+                                                const void* v_cache, const uint64_t* mask_dev, int32_t n,
+                                                int32_t kv_len, void* out, char* err_buf, size_t err_len) {
+    using namespace ghd;
+    if (!q || !k_cache || !v_cache || !mask_dev || !out) { st_error(err_buf, err_len, "null pointer argument"); return GHD_EINVAL; }
+    if (dtype != GHD_F32 && dtype != GHD_F16) { st_error(err_buf, err_len, "dtype must be GHD_F32 or GHD_F16"); return GHD_EINVAL; }
+    if (d_head != 64 && d_head != 128) { st_error(err_buf, err_len, "d_head must be 64 or 128"); return GHD_ESHAPE; }
+    if (n_heads < 1 || n < 1 || kv_len < 0 || max_kv_len < 1) { st_error(err_buf, err_len, "non-positive size"); return GHD_EINVAL; }
+    if (n > ST_MAX_NODES || (int64_t)n_heads * d_head > ST_MAX_WIDTH) {
+        st_error(err_buf, err_len, "beyond the built-in scratch: at most 64 tree nodes and n_heads * d_head <= 4096");
+        return GHD_ENOSPACE;
+    }
+    if ((int64_t)kv_len + n > max_kv_len) { st_error(err_buf, err_len, "kv_len + n > max_kv_len"); return GHD_ENOSPACE; }
+
+    // Set-up, once per device: in host code `g_static_scratch` is only a handle of the
+    // symbol, so ask the runtime where the array lives on the current device.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= ST_MAX_DEVICES) {
+        st_error(err_buf, err_len, "cannot identify the current device");
+        return GHD_ECUDA;
+    }
+    float* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> hold(g_static_scratch_lock);
+        if (!g_static_scratch_addr[dev]) {
+            void* p = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+            if (e != cudaSuccess || !p) {
+                st_error(err_buf, err_len, cudaGetErrorString(e));
+                return GHD_ECUDA;
+            }
+            g_static_scratch_addr[dev] = static_cast<float*>(p);
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    float* part_o = scratch;
+    float* part_ml = scratch + ST_O_FLOATS;
+
+    // Nothing in the array has to start at zero: every (split, node, head) slot that the merge
+    // kernel reads is written by the split kernel of this same call (splits without a visible
+    // key write max = -inf, sum = 0), so what an earlier call left behind is never observed.
+    const int kt = kv_len + n;
+    int splits = (kt + 255) / 256;
+    if (splits > ST_MAX_SPLITS) splits = ST_MAX_SPLITS;
+    if (splits < 1) splits = 1;
+    int chunk = (kt + splits - 1) / splits;
+    chunk = ((chunk + TK - 1) / TK) * TK;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    dim3 grid((n + QB - 1) / QB, n_heads, splits);
+    const int n_words = (n + 63) / 64;
+#define GHD_ATTN_ST(T, DH)                                                                                  \
+    k_attn_simt<T, DH><<<grid, QB * 32, 0, stream>>>((const T*)q, (const T*)k_cache, (const T*)v_cache,      \
+                                                     mask_dev, n_words, n, n_heads, kv_len, max_kv_len,      \
+                                                     chunk, part_o, part_ml, ST_MAX_NODES)
+    if (dtype == GHD_F32) { if (d_head == 64) GHD_ATTN_ST(float, 64); else GHD_ATTN_ST(float, 128); }
+    else { if (d_head == 64) GHD_ATTN_ST(__half, 64); else GHD_ATTN_ST(__half, 128); }
+#undef GHD_ATTN_ST
+    dim3 cgrid(n, n_heads);
+    if (dtype == GHD_F32)
+        k_attn_combine<float><<<cgrid, d_head, 0, stream>>>(part_o, part_ml, (float*)out, splits, n_heads, d_head, ST_MAX_NODES);
+    else
+        k_attn_combine<__half><<<cgrid, d_head, 0, stream>>>(part_o, part_ml, (__half*)out, splits, n_heads, d_head, ST_MAX_NODES);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { st_error(err_buf, err_len, cudaGetErrorString(e)); return GHD_ECUDA; }
+    return GHD_OK;
+}
