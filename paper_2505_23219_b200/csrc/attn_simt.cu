@@ -164,6 +164,18 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
     c->launches++;
 }
 
+void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n) {
+    const ghd_model_cfg& m = c->cfg;
+    dim3 cgrid(n, m.n_heads);
+    if (m.dtype == GHD_F32)
+        k_attn_combine<float><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (float*)out, splits, m.n_heads,
+                                                              m.d_head, m.max_nodes);
+    else
+        k_attn_combine<__half><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (__half*)out, splits, m.n_heads,
+                                                               m.d_head, m.max_nodes);
+    c->launches++;
+}
+
 // ---------------------------------------------------------------------------
 // Tree attention for callers that cannot allocate device memory.
 //

@@ -1,0 +1,394 @@
+// Tree attention on the tensor cores (sm_100a, half in, float softmax/accumulate).
+//
+// One CTA = one head x one tile of up to 128 query nodes x one KV split.  Keys are
+// walked in 64-key units: the cache rows [0, kv_len) first (the dense part: every
+// query sees every row), then the new rows in groups of 64 nodes = one word of the
+// packed ancestor bitmask per query (the sparse part).  A node group whose mask
+// word is zero for every query of the CTA is dropped from the unit list before
+// anything is loaded.  The units are divided evenly among the splits of a head.
+//
+// Per unit:  S = Q K^T   (tcgen05.mma, Q and K tile K-major in swizzled shared memory,
+//                         S [128 x 64] float in tensor memory)
+//            softmax warps (one thread per query row) read S, apply the mask, keep a
+//            running (max, sum), and write P = exp(S - max) as half into shared memory
+//            PV = P V     (tcgen05.mma, V tile consumed row-major as an N-major operand)
+//            softmax warps fold PV into their float output registers, rescaled by
+//            exp(old max - new max)
+// S and PV are double-buffered in tensor memory so that S of unit j+1 is computed
+// while unit j is in softmax.  Each CTA writes un-normalised (o, max, sum) for its
+// split; k_attn_combine merges the splits (paper Sec. III-B-2: per-partition
+// softmax aligned by a scaling factor at the end).
+//
+// Warp 0 = TMA producer, warp 1 = MMA issuer + tensor-memory owner, warps 2..5 =
+// softmax (128 threads = 128 tensor-memory lanes).  All waits are bounded.
+#include <cstdio>
+
+#include "internal.h"
+#include "tc_common.cuh"
+
+namespace ghd {
+
+namespace {
+
+using namespace tc;
+
+constexpr int QM = 128;        // query rows per CTA (MMA M)
+constexpr int BN = 64;         // keys per unit (MMA N of S, MMA K of PV)
+constexpr int KV_STAGES = 4;
+constexpr int THREADS = 192;
+constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
+
+struct AttnParams {
+    int n, heads, kv_len, max_nodes, splits, n_words;
+    const uint64_t* mask;
+    float* part_o;
+    float* part_ml;
+    int* status;
+    float scale;               // 1 / sqrt(d_head)
+};
+
+struct AttnSmem {
+    uint64_t q_full;
+    uint64_t kv_full[KV_STAGES], kv_empty[KV_STAGES];
+    uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2], pv_full[2], pv_empty[2];
+    uint64_t drain;
+    unsigned long long word_or[MAX_UNITS_WORDS];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(THREADS, 1)
+k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+          const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    constexpr int SLABS = DH / 64;                       // 64-wide (128-byte) column slabs of a d_head row
+    constexpr uint32_t Q_SLAB = QM * 128;                // bytes of one [128 x 64] half slab
+    constexpr uint32_t KV_SLAB = BN * 128;               // bytes of one [64 x 64] half slab
+    constexpr uint32_t Q_BYTES = SLABS * Q_SLAB;
+    constexpr uint32_t STAGE_BYTES = 2 * SLABS * KV_SLAB;   // K slabs then V slabs
+    constexpr uint32_t P_BYTES = QM * 128;               // [128 x 64] half
+    constexpr uint32_t TMEM_S = 0, TMEM_PV = 2 * BN;     // columns: S[2] then PV[2]
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* base = smem_raw + pad;
+    const uint32_t q_addr = smem_u32(base);
+    const uint32_t kv_addr = q_addr + Q_BYTES;
+    const uint32_t p_addr = kv_addr + KV_STAGES * STAGE_BYTES;
+    uint8_t* p_ptr = base + Q_BYTES + KV_STAGES * STAGE_BYTES;
+    AttnSmem* sm = reinterpret_cast<AttnSmem*>(p_ptr + 2 * P_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x, h = blockIdx.y, mtile = blockIdx.z;
+    const int row0 = mtile * QM;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&sm->q_full), 1);
+        for (int s = 0; s < KV_STAGES; ++s) { mbar_init(smem_u32(&sm->kv_full[s]), 1); mbar_init(smem_u32(&sm->kv_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sm->s_full[b]), 1);
+            mbar_init(smem_u32(&sm->s_empty[b]), 128);
+            mbar_init(smem_u32(&sm->p_full[b]), 128);
+            mbar_init(smem_u32(&sm->p_empty[b]), 1);
+            mbar_init(smem_u32(&sm->pv_full[b]), 1);
+            mbar_init(smem_u32(&sm->pv_empty[b]), 128);
+        }
+        mbar_init(smem_u32(&sm->drain), 1);
+        for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // which 64-node groups does any query row of this CTA see?
+    if (threadIdx.x >= 64) {
+        const int row = row0 + (int)threadIdx.x - 64;
+        if (row < p.n)
+            for (int w = 0; w < p.n_words; ++w) {
+                const unsigned long long bits = p.mask[(size_t)row * p.n_words + w];
+                if (bits) atomicOr(&sm->word_or[w], bits);
+            }
+    }
+    __syncthreads();
+    const uint32_t tmem_base = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+
+    // unit list: cache tiles, then the visible node groups; this CTA's share of it
+    const int n_cache = (p.kv_len + BN - 1) / BN;
+    uint32_t act = 0;                                    // bit w set: node group w is visible to some row
+#pragma unroll
+    for (int w = 0; w < MAX_UNITS_WORDS; ++w)
+        if (w < p.n_words && sm->word_or[w] != 0ull) act |= 1u << w;
+    const int total = n_cache + __popc(act);
+    const int u_beg = (int)((long long)total * split / p.splits), u_end = (int)((long long)total * (split + 1) / p.splits);
+    const int cnt = u_end - u_beg;
+    auto unit_word = [&](int u) -> int {                 // the (u - n_cache)-th visible node group
+        int left = u - n_cache, w = 0;
+#pragma unroll
+        for (int a = 0; a < MAX_UNITS_WORDS; ++a)
+            if ((act >> a) & 1u) { if (left == 0) w = a; --left; }
+        return w;
+    };
+    auto unit_key0 = [&](int u) -> int { return u < n_cache ? u * BN : p.kv_len + 64 * unit_word(u); };
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0 && cnt > 0) {
+            uint64_t pol_q, pol_kv;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_q));
+            if (gridDim.z > 1) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_kv));
+            else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_kv));
+            mbar_expect_tx(smem_u32(&sm->q_full), Q_BYTES);
+#pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+                tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
+            uint32_t stage = 0, phase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (int i = 0; i < cnt; ++i) {
+                if (issued >= KV_STAGES) ok = mbar_wait(smem_u32(&sm->kv_empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+                if (!ok) break;
+                const int key0 = unit_key0(u_beg + i);
+                const uint32_t full = smem_u32(&sm->kv_full[stage]);
+                const uint32_t k_dst = kv_addr + stage * STAGE_BYTES, v_dst = k_dst + SLABS * KV_SLAB;
+                mbar_expect_tx(full, STAGE_BYTES);
+#pragma unroll
+                for (int s = 0; s < SLABS; ++s) {
+                    tma_load_3d(k_dst + s * KV_SLAB, &tm_k, s * 64, key0, h, full, pol_kv);
+                    tma_load_3d(v_dst + s * KV_SLAB, &tm_v, s * 64, key0, h, full, pol_kv);
+                }
+                ++issued;
+                if (++stage == KV_STAGES) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) {
+                const int inflight = issued < KV_STAGES ? issued : KV_STAGES;
+                uint32_t s = stage, ph = phase;
+                for (int q = 0; q < inflight; ++q) {
+                    if (s == 0) { s = KV_STAGES - 1; ph ^= 1; } else --s;
+                    for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->kv_full[s]), ph); ++spin) __nanosleep(64);
+                }
+                for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->q_full), 0); ++spin) __nanosleep(64);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0 && cnt > 0) {
+            const uint32_t idesc_s = instr_desc_f16(BN, false);          // S: N = 64 keys, K tile K-major
+            const uint32_t idesc_pv = instr_desc_f16(64, true);          // PV: N = 64 of d_head, V is N-major
+            bool ok = mbar_wait(smem_u32(&sm->q_full), 0, abort_flag, p.status, DEV_TIMEOUT_MMA);
+            tc_fence_after();
+            auto issue_pv = [&](int i) -> bool {
+                const int b = i & 1, stage = i % KV_STAGES;
+                if (!mbar_wait(smem_u32(&sm->p_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) return false;
+                if (i >= 2 && !mbar_wait(smem_u32(&sm->pv_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM)) return false;
+                tc_fence_after();
+                const uint32_t v_addr = kv_addr + stage * STAGE_BYTES + SLABS * KV_SLAB;
+                const uint64_t pdesc = smem_desc_sw128(p_addr + b * P_BYTES);
+#pragma unroll
+                for (int s = 0; s < SLABS; ++s) {
+                    const uint32_t d_tmem = tmem_base + TMEM_PV + b * DH + s * 64;
+#pragma unroll
+                    for (int ks = 0; ks < BN / 16; ++ks)     // 16 keys per MMA: +32 B along P's rows, +16 rows of V
+                        tc_mma_f16(d_tmem, pdesc + (uint64_t)(ks * 2), smem_desc_sw128(v_addr + s * KV_SLAB + ks * 16 * 128),
+                                   idesc_pv, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(smem_u32(&sm->pv_full[b]));
+                tc_commit(smem_u32(&sm->kv_empty[stage]));
+                tc_commit(smem_u32(&sm->p_empty[b]));
+                return true;
+            };
+            for (int i = 0; i < cnt && ok; ++i) {
+                const int b = i & 1, stage = i % KV_STAGES;
+                ok = mbar_wait(smem_u32(&sm->kv_full[stage]), (i / KV_STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA);
+                if (ok && i >= 2) ok = mbar_wait(smem_u32(&sm->s_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t k_addr = kv_addr + stage * STAGE_BYTES;
+                const uint32_t d_tmem = tmem_base + TMEM_S + b * BN;
+#pragma unroll
+                for (int s = 0; s < SLABS; ++s)
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        tc_mma_f16(d_tmem, smem_desc_sw128(q_addr + s * Q_SLAB) + (uint64_t)(ks * 2),
+                                   smem_desc_sw128(k_addr + s * KV_SLAB) + (uint64_t)(ks * 2), idesc_s, (s > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&sm->s_full[b]));
+                if (i >= 1) ok = issue_pv(i - 1);
+            }
+            if (ok) ok = issue_pv(cnt - 1);
+            if (!ok) {
+                tc_commit(smem_u32(&sm->drain));
+                for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain), 0); ++spin) __nanosleep(64);
+            }
+        }
+    } else {
+        // ------------------------------------------------ softmax warps: thread = query row
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                        // row inside the tile = tensor-memory lane
+        const int row = row0 + r;
+        const bool live = row < p.n;
+        const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+        const float c_log2e = 1.4426950408889634f;
+        float m = -INFINITY, l = 0.f, corr_prev = 1.f;
+        float o[DH];
+#pragma unroll
+        for (int c = 0; c < DH; ++c) o[c] = 0.f;
+
+        auto fold_pv = [&](int i, float corr) {
+            const int b = i & 1;
+            mbar_wait(smem_u32(&sm->pv_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < DH; c0 += 32) {
+                float v[32];
+                tc_ld32(tmem_base + TMEM_PV + b * DH + c0 + lane_off, v);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&sm->pv_empty[b]));
+        };
+
+        for (int i = 0; i < cnt; ++i) {
+            const int u = u_beg + i, b = i & 1;
+            // visibility of the 64 keys of this unit for this row
+            unsigned long long vis = 0ull;
+            if (live) {
+                if (u < n_cache) {
+                    const int valid = p.kv_len - u * BN;
+                    vis = valid >= 64 ? ~0ull : ((1ull << valid) - 1ull);
+                } else {
+                    vis = p.mask[(size_t)row * p.n_words + unit_word(u)];
+                }
+            }
+            mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            tc_fence_after();
+            float s[BN];
+            {
+                float t[32];
+                tc_ld32(tmem_base + TMEM_S + b * BN + lane_off, t);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) s[j] = t[j];
+                tc_ld32(tmem_base + TMEM_S + b * BN + 32 + lane_off, t);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) s[32 + j] = t[j];
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&sm->s_empty[b]));
+            float tmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < BN; ++j) {
+                s[j] *= p.scale;
+                if ((vis >> j) & 1ull) tmax = fmaxf(tmax, s[j]);
+            }
+            const float m_new = fmaxf(m, tmax);
+            float corr = 1.f, psum = 0.f;
+            const float mb = (m_new == -INFINITY) ? 0.f : m_new * c_log2e;
+            if (m_new != -INFINITY) corr = (m == -INFINITY) ? 0.f : exp2f(m * c_log2e - mb);
+            // P row -> shared memory, K-major with the 128-byte swizzle the MMA descriptor expects
+            if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            uint8_t* prow = p_ptr + b * P_BYTES + r * 128;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                uint32_t packed[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int j = ch * 8 + 2 * e;
+                    const float p0 = ((vis >> j) & 1ull) ? exp2f(fmaf(s[j], c_log2e, -mb)) : 0.f;
+                    const float p1 = ((vis >> (j + 1)) & 1ull) ? exp2f(fmaf(s[j + 1], c_log2e, -mb)) : 0.f;
+                    const __half2 hh = __floats2half2_rn(p0, p1);
+                    psum += __low2float(hh) + __high2float(hh);
+                    packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(smem_u32(&sm->p_full[b]));
+            l = l * corr + psum;
+            m = m_new;
+            if (i >= 1) fold_pv(i - 1, corr_prev);
+            corr_prev = corr;
+        }
+        if (cnt > 0) fold_pv(cnt - 1, corr_prev);
+        if (live) {
+            float* po = p.part_o + ((size_t)split * p.max_nodes + row) * (size_t)(p.heads * DH) + h * DH;
+#pragma unroll
+            for (int c = 0; c < DH; c += 4) *reinterpret_cast<float4*>(po + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+            float* pm = p.part_ml + (((size_t)split * p.max_nodes + row) * p.heads + h) * 2;
+            pm[0] = m;
+            pm[1] = l;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+template <int DH>
+size_t attn_smem_bytes() {
+    return 1024 + (size_t)(DH / 64) * QM * 128 + (size_t)KV_STAGES * 2 * (DH / 64) * BN * 128 + 2 * QM * 128 + sizeof(AttnSmem);
+}
+
+}  // namespace
+
+bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t) {
+    return c->cfg.dtype == GHD_F16 && (c->cfg.d_head == 64 || c->cfg.d_head == 128) && t->n >= 1;
+}
+
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
+    const ghd_model_cfg& m = c->cfg;
+    const int n = t->n, H = m.n_heads, dh = m.d_head, d = m.d_model;
+    const int kt = t->kv_len + n;
+    if (((uintptr_t)q & 15) || ((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15)) {
+        snprintf(c->err, sizeof(c->err), "tcgen05 attention: operands must be 16-byte aligned");
+        return GHD_EINVAL;
+    }
+    CUtensorMap tm_q, tm_k, tm_v;
+    if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, QM, &tm_q) ||
+        !tmap_planes(c, kv->k, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_k) ||
+        !tmap_planes(c, kv->v, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_v)) {
+        snprintf(c->err, sizeof(c->err), "tcgen05 attention: tensor map encoding failed");
+        return GHD_ECUDA;
+    }
+    const int mtiles = (n + QM - 1) / QM;
+    const int units = (t->kv_len + BN - 1) / BN + t->n_words;
+    int splits = c->opt_attn_splits;
+    if (splits <= 0) {
+        splits = c->sm_count / (H * mtiles);
+        const int by_len = (units + 1) / 2;              // at least two units per split
+        if (splits > by_len) splits = by_len;
+    }
+    if (splits > c->max_splits) splits = c->max_splits;
+    if (splits < 1) splits = 1;
+    AttnParams p{};
+    p.n = n; p.heads = H; p.kv_len = t->kv_len; p.max_nodes = m.max_nodes; p.splits = splits; p.n_words = t->n_words;
+    p.mask = t->mask; p.part_o = c->att_o; p.part_ml = c->att_ml; p.status = c->status;
+    p.scale = 1.0f / sqrtf((float)dh);
+    dim3 grid(splits, H, mtiles);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<64>()) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<128>()) != cudaSuccess) {
+            snprintf(c->err, sizeof(c->err), "tcgen05 attention: cannot raise dynamic shared memory");
+            cudaGetLastError();
+            return GHD_ECUDA;
+        }
+        attr_set = true;
+    }
+    if (dh == 64) k_attn_tc<64><<<grid, THREADS, attn_smem_bytes<64>(), c->cur>>>(tm_q, tm_k, tm_v, p);
+    else k_attn_tc<128><<<grid, THREADS, attn_smem_bytes<128>(), c->cur>>>(tm_q, tm_k, tm_v, p);
+    c->launches++;
+    launch_attn_combine(c, out, splits, n);
+    return GHD_OK;
+}
+
+}  // namespace ghd

@@ -350,46 +350,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
-// Row-major half matrix [rows][cols] -> tensor map with a (box_rows x 64) box, 128-byte swizzle, zero fill.
-bool get_tmap(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
-    TmapKey key{ptr, rows, cols, box_rows, (uint32_t)TILE_K};
-    auto it = c->tmaps->find(key);
-    if (it != c->tmaps->end()) { memcpy(out, it->second.data(), sizeof(CUtensorMap)); return true; }
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)TILE_K, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUtensorMap tm;
-    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    std::vector<uint64_t> blob(sizeof(CUtensorMap) / 8);
-    memcpy(blob.data(), &tm, sizeof(CUtensorMap));
-    if (c->tmaps->size() > 4096) c->tmaps->clear();
-    (*c->tmaps)[key] = blob;
-    *out = tm;
-    return true;
-}
-
 size_t smem_bytes_for(int nb, int stages) {
     return 1024 + (size_t)stages * (TILE_M * TILE_K * 2 + (size_t)nb * TILE_K * 2) + sizeof(Smem);
 }
@@ -430,8 +390,8 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     p.status = c->status;
     p.epi = epi;
     CUtensorMap tm_w, tm_x;
-    if (!get_tmap(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 64 : TILE_M, &tm_w) ||
-        !get_tmap(c, x, (uint64_t)n, (uint64_t)k, (uint32_t)p.nb, &tm_x)) {
+    if (!tmap_rows_x_k(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 64 : TILE_M, &tm_w) ||
+        !tmap_rows_x_k(c, x, (uint64_t)n, (uint64_t)k, (uint32_t)p.nb, &tm_x)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: tensor map encoding failed");
         return GHD_ECUDA;
     }

@@ -75,7 +75,9 @@ static ghd_status project(ghd_ctx* c, const void* x, const void* w, int n, int k
 }
 
 static ghd_status attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
-    if (c->opt_attn_path == 2) return fail(c, GHD_EUNSUPPORTED, "tcgen05 attention is not built");
+    const bool tc_ok = attn_tc_supported(c, t);
+    if (c->opt_attn_path == 2 && !tc_ok) return fail(c, GHD_EUNSUPPORTED, "tcgen05 attention does not take this type/shape");
+    if (tc_ok && c->opt_attn_path != 1) return launch_attn_tc(c, q, kv, t, out);
     launch_attn_simt(c, q, kv, t, out);
     return GHD_OK;
 }

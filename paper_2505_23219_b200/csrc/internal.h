@@ -35,9 +35,10 @@ struct EpiArgs {
 };
 
 struct TmapKey {
-    const void* ptr; uint64_t rows, cols; uint32_t box_rows, box_cols;
+    const void* ptr; uint64_t rows, cols, planes, plane_stride; uint32_t box_rows, box_cols;
     bool operator<(const TmapKey& o) const {
-        return std::tie(ptr, rows, cols, box_rows, box_cols) < std::tie(o.ptr, o.rows, o.cols, o.box_rows, o.box_cols);
+        return std::tie(ptr, rows, cols, planes, plane_stride, box_rows, box_cols) <
+               std::tie(o.ptr, o.rows, o.cols, o.planes, o.plane_stride, o.box_rows, o.box_cols);
     }
 };
 
@@ -99,6 +100,12 @@ void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, in
 // attn_simt.cu : split-KV tree attention + combine
 void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
 int attn_auto_splits(const ghd_ctx* c, int n, int kv_total);
+
+void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n);   // merges att_o / att_ml into out
+
+// attn_tc.cu : tcgen05 / TMA tree attention (GHD_F16 only)
+bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t);
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
 
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);

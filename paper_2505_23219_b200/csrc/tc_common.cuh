@@ -107,5 +107,21 @@ __device__ __forceinline__ uint32_t instr_desc_f16(int nb, bool b_mn_major = fal
 }
 
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy) : "memory");
+}
+
 }  // namespace tc
+
+// Host: cached tensor maps (half elements, 128-byte swizzle, 64-element inner box, zero fill).
+// Row-major matrix [rows][cols] with a (box_rows x 64) box.
+bool tmap_rows_x_k(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out);
+// [planes][rows_alloc][cols] of which only the first `rows` rows of each plane are readable
+// (rows beyond read as zero); box = (1 plane x box_rows x 64).
+bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
+                 uint32_t box_rows, CUtensorMap* out);
+
 }  // namespace ghd

@@ -154,9 +154,11 @@ def test_linear_tcgen05_path(ghd, n, k, m):
         assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
 
 
-def _attention_case(ghd, shape, n, L, parent, splits, seed=400):
+def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0):
     Lmax = L + n + 3
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
+    if path:
+        ghd.ghd_set_option(ctx, ghd.OPT_ATTN_PATH, path)
     if splits:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPLITS, splits)
     H, dh, dt = shape.n_heads, shape.d_head, shape.dtype
@@ -185,9 +187,17 @@ def test_tree_attention(ghd, shape, n, L, splits):
     assert err <= (2e-5 if shape.dtype == "f32" else 2e-3)
 
 
+@pytest.mark.parametrize("n,L,splits", [(64, 2048, 0), (64, 2048, 5), (200, 1000, 0), (256, 4096, 0), (49, 640, 3)])
+def test_tree_attention_long_cache_both_paths(ghd, n, L, splits):
+    parent = wl.random_tree(n, 8, 2000 + n, max_children=6)
+    assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits) <= 2e-3               # tcgen05 kernel
+    assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits, path=1) <= 2e-3       # CUDA-core kernel
+
+
 def test_chain_tree_is_causal_attention_and_star_sees_only_root(ghd):
     for parent in (wl.chain_tree(40), wl.star_tree(40)):
         assert _attention_case(ghd, SMALL32, 40, 50, parent, 0) <= 2e-5
+        assert _attention_case(ghd, SMALL16, 40, 50, parent, 0) <= 2e-3
 
 
 def test_argmax_bit_exact_including_ties(ghd):
