@@ -54,7 +54,8 @@ typedef enum ghd_option {
     GHD_OPT_ATTN_PATH = 2,    /* 0 auto, 1 SIMT kernel, 2 tcgen05 kernel (GHD_F16 only)      */
     GHD_OPT_GRAPH = 3,        /* ghd_verify_step: 0/1 = launch kernels directly, 2 = replay a
                                  CUDA graph captured on first use for the same arguments    */
-    GHD_OPT_GEMM_CTAS = 4     /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
+    GHD_OPT_GEMM_CTAS = 4,    /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
+    GHD_OPT_GEMM_BURST = 5    /* k-steps whose weight loads the tcgen05 GEMM issues together  */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary

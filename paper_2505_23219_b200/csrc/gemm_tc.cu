@@ -43,6 +43,7 @@ constexpr int THREADS = 192;
 struct GemmParams {
     int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
     int n_tiles, kiters, stages;
+    int burst;                       // k-steps whose loads are issued back to back (adjacent 128-byte chunks of the same weight rows)
     int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
     float* part;                     // [ctas][2][nb][128] float partial tiles
     int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
@@ -80,14 +81,19 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
     if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
         const int f = tile * TILE_M + row;
         if (f < p.m) {
+            float* dst = e.out_f32 + (size_t)c0 * p.m + f;
+            if (e.mode == EPI_RESID) {
+                // all loads first, then all stores: a load placed after a store through another
+                // pointer would have to wait for it, turning 32 round trips into a chain
+                float old[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int node = c0 + j;
-                if (node < p.n) {
-                    float* dst = e.out_f32 + (size_t)node * p.m + f;
-                    *dst = (e.mode == EPI_RESID) ? (*dst + v[j]) : v[j];
-                }
+                for (int j = 0; j < 32; ++j) old[j] = (c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.m) : 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] += old[j];
             }
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (c0 + j < p.n) dst[(size_t)j * p.m] = v[j];
         }
         return;
     }
@@ -122,18 +128,24 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
         epi_bar();
         const int prow = (idx < half) ? row + half : row - half;
         const int t = (idx < half) ? idx : idx - half;
+        const float sign = (idx < half) ? -1.f : 1.f;
+        float2 cs[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int node = c0 + j;
-            if (node < p.n) {
-                const float2 cs = *reinterpret_cast<const float2*>(e.rope + (size_t)node * dh + 2 * t);
-                const float other = sm->stage_x[j][prow];
-                const float r = (idx < half) ? (v[j] * cs.x - other * cs.y) : (v[j] * cs.x + other * cs.y);
-                if (section == 0)
-                    ((__half*)e.out_t)[(size_t)node * d + el] = __float2half_rn(r);
-                else
-                    ((__half*)e.k_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(r);
-            }
+        for (int j = 0; j < 32; ++j)       // table loads before any store (see above)
+            cs[j] = (c0 + j < p.n) ? __ldg(reinterpret_cast<const float2*>(e.rope + (size_t)(c0 + j) * dh + 2 * t)) : make_float2(1.f, 0.f);
+        float r[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
+        if (section == 0) {
+            __half* qo = (__half*)e.out_t + (size_t)c0 * d + el;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (c0 + j < p.n) qo[(size_t)j * d] = __float2half_rn(r[j]);
+        } else {
+            __half* ko = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (c0 + j < p.n) ko[(size_t)j * dh] = __float2half_rn(r[j]);
         }
         epi_bar();
     } else {
@@ -193,11 +205,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             uint32_t stage = 0, phase = 0;
-            long long issued = 0;
+            int issued = 0;
             bool ok = true;
-            for (long long it = it_beg; it < it_end && ok; ++it) {
-                const int tile = (int)(it / p.kiters), kk = (int)(it - (long long)tile * p.kiters);
-                if (issued >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+            // (tile, kk) advance incrementally: a 64-bit division per k-step would cost this single
+            // thread more cycles than the loads it issues
+            int tile = (int)(it_beg / p.kiters), kk = (int)(it_beg - (long long)tile * p.kiters);
+            const int my_iters = (int)(it_end - it_beg);
+            int burst_left = 0;
+            for (int i = 0; i < my_iters && ok; ++i) {
+                if (burst_left == 0) {
+                    // free the ring slots of a whole burst first, then issue its loads together
+                    uint32_t s2 = stage, ph2 = phase;
+                    for (int j = 0; j < p.burst && i + j < my_iters && ok; ++j) {
+                        if (issued + j >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[s2]), ph2 ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+                        if (++s2 == (uint32_t)p.stages) { s2 = 0; ph2 ^= 1; }
+                    }
+                    burst_left = p.burst;
+                }
+                --burst_left;
                 if (!ok) break;
                 const uint32_t full = smem_u32(&sm->full[stage]);
                 const uint32_t a_dst = tiles_addr + stage * stage_bytes, b_dst = a_dst + a_bytes;
@@ -211,12 +236,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 tma_load_2d(b_dst, &tm_x, kk * TILE_K, 0, full, pol_keep);
                 ++issued;
                 if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                if (++kk == p.kiters) { kk = 0; ++tile; }
             }
             if (!ok) {
                 // drain: wait (bounded) until every load issued into the ring has landed
-                const long long inflight = issued < p.stages ? issued : p.stages;
+                const int inflight = issued < p.stages ? issued : p.stages;
                 uint32_t s = stage, ph = phase;
-                for (long long q = 0; q < inflight; ++q) {
+                for (int q = 0; q < inflight; ++q) {
                     if (s == 0) { s = p.stages - 1; ph ^= 1; } else --s;
                     for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->full[s]), ph); ++spin) __nanosleep(64);
                 }
@@ -270,12 +296,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
         long long it = it_beg;
-        const size_t slot_elems = (size_t)p.nb * TILE_M;
+        const size_t slot_elems = (size_t)buf_cols * TILE_M;   // columns padded to whole 32-wide chunks
         while (it < it_end && ok) {
             const int tile = (int)(it / p.kiters), k0 = (int)(it - (long long)tile * p.kiters);
             const long long left = it_end - it;
             const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
-            const bool whole = (k0 == 0 && k1 == p.kiters);
+            const bool whole = (k0 == 0 && k1 == p.kiters) && p.epi.mode != EPI_DEFER;
             mbar_wait(smem_u32(&sm->tmem_full[buf]), buf_phase, abort_flag, p.status, DEV_TIMEOUT_EPI);
             epi_bar();                                         // all 128 threads take the same decision
             ok = (*abort_flag == 0);
@@ -300,12 +326,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     float v[32];
                     tc_ld32(t_addr + c0, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c0 + j < p.nb) mine[(size_t)(c0 + j) * TILE_M + row] = v[j];
+                    for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+                if (p.epi.mode == EPI_DEFER) {                 // the consumer kernel sums the partial tiles
+                    if (++buf == 2) { buf = 0; buf_phase ^= 1; }
+                    it += (k1 - k0);
+                    continue;
+                }
                 __threadfence();
                 epi_bar();
                 const long long t_first = (long long)tile * p.kiters;
@@ -323,13 +353,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                         float v[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        // contributors in CTA order; each one's 32 loads are issued together
                         for (int c = c_first; c <= c_last; ++c) {
                             const long long cb = total * c / G;
                             const int cslot = (cb >= t_first) ? 0 : 1;
-                            const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems;
+                            const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems + (size_t)c0 * TILE_M + row;
+                            float t[32];
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (c0 + j < p.nb) v[j] += __ldcg(src + (size_t)(c0 + j) * TILE_M + row);
+                            for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * TILE_M);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += t[j];
                         }
                         epilogue_chunk(p, sm, tile, row, c0, v);
                     }
@@ -368,6 +401,12 @@ bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
     if (n_tiles < 1 || n_tiles > 4096) return false;
     if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
     if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
+    if (epi_mode == EPI_DEFER) {
+        int ctas = c->opt_gemm_ctas > 0 && c->opt_gemm_ctas < c->sm_count ? c->opt_gemm_ctas : c->sm_count;
+        const long long total = (long long)n_tiles * ((k + TILE_K - 1) / TILE_K);
+        if (ctas > total) ctas = (int)total;
+        if (m % 4 || m > 16384 || total / ctas + 1 > (k + TILE_K - 1) / TILE_K) return false;
+    }
     return true;
 }
 
@@ -385,6 +424,8 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     p.n_tiles = p.swiglu_f ? p.swiglu_f / 64 : (m + TILE_M - 1) / TILE_M;
     p.kiters = (k + TILE_K - 1) / TILE_K;
     p.stages = pick_stages(p.nb);
+    p.burst = c->opt_gemm_burst > 0 ? c->opt_gemm_burst : 1;
+    if (p.burst > p.stages / 2) p.burst = p.stages / 2 > 0 ? p.stages / 2 : 1;
     p.part = c->gemm_part;
     p.counters = c->counters;
     p.status = c->status;
@@ -407,6 +448,18 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
             return GHD_ECUDA;
         }
         attr_set = true;
+    }
+    if (epi.mode == EPI_DEFER) {
+        if (total / ctas + 1 > p.kiters) {                // a CTA range must touch at most two tiles
+            snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: deferred reduction needs n_tiles <= CTAs");
+            return GHD_EUNSUPPORTED;
+        }
+        c->pending.active = 1;
+        c->pending.kiters = p.kiters;
+        c->pending.ctas = ctas;
+        c->pending.total = total;
+        c->pending.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
+        c->pending.m = m;
     }
     k_gemm_tc<<<ctas, THREADS, smem, c->cur>>>(tm_w, tm_x, p);
     c->launches++;

@@ -74,6 +74,24 @@ static ghd_status project(ghd_ctx* c, const void* x, const void* w, int n, int k
     return GHD_OK;
 }
 
+// RMSNorm of the residual stream into hbuf, first folding in a projection whose reduction was deferred.
+static void norm_into_h(ghd_ctx* c, const void* gain, int n) {
+    if (c->pending.active) launch_fold_pending(c, n, gain, c->hbuf, nullptr);
+    else launch_rmsnorm(c, c->xres, gain, n, c->hbuf);
+}
+
+// Projection whose result is added to the residual stream.  On the tcgen05 path the k-split partial
+// tiles are left in the workspace and the next norm kernel sums them (no CTA waits, no fix-up pass).
+static ghd_status project_residual(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, EpiArgs e,
+                                   const ghd_tree* t, const ghd_kv_layer* kv) {
+    if (c->cfg.dtype == GHD_F16 && c->opt_gemm_path != 1 && gemm_tc_supported(c, n, k, m, EPI_DEFER)) {
+        e.mode = EPI_DEFER;
+        return launch_gemm_tc(c, x, w, n, k, m, e);
+    }
+    e.mode = EPI_RESID; e.out_f32 = c->xres;
+    return project(c, x, w, n, k, m, e, t, kv);
+}
+
 static ghd_status attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
     const bool tc_ok = attn_tc_supported(c, t);
     if (c->opt_attn_path == 2 && !tc_ok) return fail(c, GHD_EUNSUPPORTED, "tcgen05 attention does not take this type/shape");
@@ -88,17 +106,15 @@ static ghd_status layer_body(ghd_ctx* c, const ghd_layer_weights* w, const ghd_k
     ghd_status s;
     EpiArgs e{};
     e.rope = t->rope; e.kv_len = t->kv_len; e.max_kv_len = m.max_kv_len; e.d_head = m.d_head; e.d_model = d;
-    launch_rmsnorm(c, c->xres, w->rms1, n, c->hbuf);
+    norm_into_h(c, w->rms1, n);
     e.mode = EPI_ROPE_KV; e.out_t = c->qbuf; e.k_cache = kv->k; e.v_cache = kv->v;
     if ((s = project(c, c->hbuf, w->wqkv, n, d, 3 * d, e, t, kv)) != GHD_OK) return s;
     if ((s = attention(c, c->qbuf, kv, t, c->attnbuf)) != GHD_OK) return s;
-    e.mode = EPI_RESID; e.out_f32 = c->xres;
-    if ((s = project(c, c->attnbuf, w->wo, n, d, d, e, t, kv)) != GHD_OK) return s;
-    launch_rmsnorm(c, c->xres, w->rms2, n, c->hbuf);
+    if ((s = project_residual(c, c->attnbuf, w->wo, n, d, d, e, t, kv)) != GHD_OK) return s;
+    norm_into_h(c, w->rms2, n);
     e.mode = EPI_SWIGLU; e.out_t = c->ubuf;
     if ((s = project(c, c->hbuf, w->w_gate_up, n, d, 2 * f, e, t, kv)) != GHD_OK) return s;
-    e.mode = EPI_RESID; e.out_f32 = c->xres;
-    if ((s = project(c, c->ubuf, w->w_down, n, f, d, e, t, kv)) != GHD_OK) return s;
+    if ((s = project_residual(c, c->ubuf, w->w_down, n, f, d, e, t, kv)) != GHD_OK) return s;
     return GHD_OK;
 }
 
@@ -109,7 +125,7 @@ static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer
     launch_embed(c, w->embed, tokens, t->n);
     for (int l = 0; l < m.n_layers; ++l)
         if ((s = layer_body(c, &w->layers[l], &kv[l], t)) != GHD_OK) return s;
-    launch_rmsnorm(c, c->xres, w->rms_final, t->n, c->hbuf);
+    norm_into_h(c, w->rms_final, t->n);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = logits;
     if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
@@ -145,10 +161,11 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
+    c->pending.active = 0;
     c->launches = 0;
     c->tmaps = new std::map<TmapKey, std::vector<uint64_t>>();
     c->graphs = new std::vector<StepGraph*>();
@@ -192,6 +209,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_ATTN_PATH: if (value > 2) return GHD_EINVAL; c->opt_attn_path = value; break;
         case GHD_OPT_GRAPH: if (value > 2) return GHD_EINVAL; c->opt_graph = value; break;
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
+        case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
         default: return GHD_EINVAL;
     }
     return GHD_OK;
@@ -253,9 +271,11 @@ ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer
     ghd_status s = check_tree(c, tree);
     if (s != GHD_OK) return s;
     if (kv->len != tree->kv_len) return fail(c, GHD_EINVAL, "layer: kv.len differs from tree.kv_len");
+    c->pending.active = 0;
     launch_load_x(c, x_in, tree->n);
     if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
-    launch_store_x(c, x_out, tree->n);
+    if (c->pending.active) launch_fold_pending(c, tree->n, nullptr, nullptr, x_out);
+    else launch_store_x(c, x_out, tree->n);
     return check_cuda(c, "verify_layer");
 }
 
@@ -274,6 +294,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
         if (kv[l].len != tree->kv_len) return fail(c, GHD_EINVAL, "step: kv.len differs from tree.kv_len");
     }
     float* logits = logits_dev ? logits_dev : c->logits;
+    c->pending.active = 0;
     if (c->opt_graph != 2) {
         if ((s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev)) != GHD_OK) return s;
         return check_cuda(c, "verify_step");
@@ -285,7 +306,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
     key.push_back(((uint64_t)(uint32_t)c->opt_gemm_path << 48) | ((uint64_t)(uint32_t)c->opt_attn_splits << 32) |
-                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | (uint32_t)c->opt_gemm_ctas);
+                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | ((uint32_t)c->opt_gemm_ctas & 0xfff) | ((uint32_t)c->opt_gemm_burst << 12));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
         push(lw.wqkv); push(lw.wo); push(lw.w_gate_up); push(lw.w_down); push(lw.rms1); push(lw.rms2);

@@ -22,6 +22,7 @@ enum Epilogue : int {
     EPI_ROPE_KV = 1,  // q rotated -> q buffer; k rotated, v -> cache rows kv_len + i
     EPI_RESID = 2,    // xres[n][m] += acc (float residual stream)
     EPI_SWIGLU = 3,   // u T [n][m/2] = SiLU(gate) * up, weight rows [gate | up]
+    EPI_DEFER = 4,    // partial tiles only; the next kernel adds them to the residual stream
 };
 
 struct EpiArgs {
@@ -44,6 +45,15 @@ struct TmapKey {
 
 struct StepGraph;
 
+// Partial tiles left behind by a projection in EPI_DEFER mode: CTA c holds k-steps
+// [total*c/ctas, total*(c+1)/ctas) of the flattened (tile, k-step) space; its first unit is in
+// slot 0, its second (if any) in slot 1, each slot [columns][128 rows] float.
+struct PendingPartials {
+    int active, kiters, ctas, m;
+    long long total;
+    size_t slot_elems;
+};
+
 }  // namespace ghd
 
 struct ghd_ctx {
@@ -53,7 +63,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -70,6 +80,7 @@ struct ghd_ctx {
     float* logits;    // float [max_nodes][vocab]
     int* status;      // device status word
     int max_splits;
+    ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
     int64_t launches;
     char err[256];
@@ -88,6 +99,8 @@ void launch_load_x(ghd_ctx* c, const void* x_in, int n);     // T [n][d] -> xres
 void launch_store_x(ghd_ctx* c, void* x_out, int n);         // xres -> T [n][d]
 void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n);
 void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out);
+// xres += sum of the pending partial tiles; then optionally h = RMSNorm(xres) * g and/or x_out = T(xres)
+void launch_fold_pending(ghd_ctx* c, int n, const void* g, void* h_out, void* x_out);
 void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, const ghd_kv_layer* kv);
 void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n);
 void launch_residual(ghd_ctx* c, const float* proj_raw, int n);

@@ -151,23 +151,136 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
     return r;
 }
 
-// One block per row: out = x * g / sqrt(mean(x^2) + eps), math in float.
+// One block per row: out = x * g / sqrt(mean(x^2) + eps), math in float.  The row is read
+// once with 16-byte loads and kept in registers (up to RMS_V float4 per thread).
+constexpr int RMS_V = 4;
+
+template <typename T> __device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<__half>(__half* p, float a, float b, float c, float d) {
+    const __half2 lo = __floats2half2_rn(a, b), hi = __floats2half2_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t*>(&lo);
+    u.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+template <typename T> __device__ __forceinline__ float4 load4(const T* p);
+template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <> __device__ __forceinline__ float4 load4<__half>(const __half* p) {
+    const uint2 u = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+
 template <typename T>
 __global__ void k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, T* __restrict__ out, int d, float eps) {
     __shared__ float red[32];
     const float* row = x + (size_t)blockIdx.x * d;
+    const int nv = d >> 2;                        // d is a multiple of 8
+    float4 v[RMS_V];
     float ss = 0.f;
-    for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x) { const float v = row[cidx]; ss += v * v; }
+#pragma unroll
+    for (int k = 0; k < RMS_V; ++k) {
+        const int idx = threadIdx.x + k * blockDim.x;
+        v[k] = (idx < nv) ? *reinterpret_cast<const float4*>(row + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+    }
+    for (int idx = threadIdx.x + RMS_V * blockDim.x; idx < nv; idx += blockDim.x) {      // very wide rows
+        const float4 w = *reinterpret_cast<const float4*>(row + 4 * idx);
+        ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+    }
     ss = block_sum(ss, red);
     const float r = rsqrtf(ss / (float)d + eps);
-    for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x)
-        out[(size_t)blockIdx.x * d + cidx] = from_f32<T>(row[cidx] * r * to_f32<T>(g[cidx]));
+    T* orow = out + (size_t)blockIdx.x * d;
+#pragma unroll
+    for (int k = 0; k < RMS_V; ++k) {
+        const int idx = threadIdx.x + k * blockDim.x;
+        if (idx < nv) {
+            const float4 gg = load4<T>(g + 4 * idx);
+            store4<T>(orow + 4 * idx, v[k].x * r * gg.x, v[k].y * r * gg.y, v[k].z * r * gg.z, v[k].w * r * gg.w);
+        }
+    }
+    for (int idx = threadIdx.x + RMS_V * blockDim.x; idx < nv; idx += blockDim.x) {
+        const float4 w = *reinterpret_cast<const float4*>(row + 4 * idx);
+        const float4 gg = load4<T>(g + 4 * idx);
+        store4<T>(orow + 4 * idx, w.x * r * gg.x, w.y * r * gg.y, w.z * r * gg.z, w.w * r * gg.w);
+    }
 }
 
 void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out) {
     const int d = c->cfg.d_model;
-    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, 256, 0, c->cur>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
-                   (k_rmsnorm<__half><<<n, 256, 0, c->cur>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
+    int threads = ((d / 4 + 31) / 32) * 32;
+    if (threads > 1024) threads = 1024;
+    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, threads, 0, c->cur>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
+                   (k_rmsnorm<__half><<<n, threads, 0, c->cur>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
+    c->launches++;
+}
+
+// Folds the partial tiles of a deferred-reduction projection into the residual stream and,
+// in the same pass, produces the next RMSNorm output.  One block per node; a thread owns four
+// consecutive features (all inside one 128-row tile), adds that tile's contributors in CTA
+// order (fixed order -> reproducible), then the row's mean square is reduced across the block.
+template <typename T>
+__global__ void k_fold_pending(float* __restrict__ xres, const float* __restrict__ part, PendingPartials pp,
+                               const T* __restrict__ g, T* __restrict__ h_out, T* __restrict__ x_out, int d, float eps) {
+    __shared__ float red[32];
+    const int node = blockIdx.x;
+    const int nv = d >> 2;
+    float4 v[RMS_V];
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < RMS_V; ++k) {
+        const int idx = threadIdx.x + k * blockDim.x;
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < nv) {
+            const int f = 4 * idx, tile = f >> 7, row = f & 127;
+            const long long t_first = (long long)tile * pp.kiters;
+            const int c_first = (int)(((t_first + 1) * pp.ctas + pp.total - 1) / pp.total) - 1;
+            const int c_last = (int)(((t_first + pp.kiters) * pp.ctas + pp.total - 1) / pp.total) - 1;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c = c_first; c <= c_last; ++c) {
+                const int slot = (pp.total * c / pp.ctas >= t_first) ? 0 : 1;
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)c * 2 + slot) * pp.slot_elems +
+                                                                        (size_t)node * 128 + row));
+                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            }
+            float4 x = *reinterpret_cast<const float4*>(xres + (size_t)node * d + f);
+            x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
+            *reinterpret_cast<float4*>(xres + (size_t)node * d + f) = x;
+            v[k] = x;
+            ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+        }
+    }
+    if (x_out) {
+#pragma unroll
+        for (int k = 0; k < RMS_V; ++k) {
+            const int idx = threadIdx.x + k * blockDim.x;
+            if (idx < nv) store4<T>(x_out + (size_t)node * d + 4 * idx, v[k].x, v[k].y, v[k].z, v[k].w);
+        }
+    }
+    if (h_out) {
+        ss = block_sum(ss, red);
+        const float r = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+        for (int k = 0; k < RMS_V; ++k) {
+            const int idx = threadIdx.x + k * blockDim.x;
+            if (idx < nv) {
+                const float4 gg = load4<T>(g + 4 * idx);
+                store4<T>(h_out + (size_t)node * d + 4 * idx, v[k].x * r * gg.x, v[k].y * r * gg.y, v[k].z * r * gg.z, v[k].w * r * gg.w);
+            }
+        }
+    }
+}
+
+void launch_fold_pending(ghd_ctx* c, int n, const void* g, void* h_out, void* x_out) {
+    const int d = c->cfg.d_model;
+    int threads = (((d / 4 + RMS_V - 1) / RMS_V + 31) / 32) * 32;      // d/4 float4 per row, up to RMS_V per thread
+    if (d / 4 <= 1024) threads = ((d / 4 + 31) / 32) * 32;
+    k_fold_pending<__half><<<n, threads, 0, c->cur>>>(c->xres, c->gemm_part, c->pending, (const __half*)g, (__half*)h_out,
+                                                      (__half*)x_out, d, c->cfg.rms_eps);
+    c->pending.active = 0;
     c->launches++;
 }
 
@@ -252,7 +365,19 @@ __global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __res
     const float* row = logits + (size_t)blockIdx.x * v;
     float best = -INFINITY;
     int bi = 0x7fffffff;
-    for (int cidx = threadIdx.x; cidx < v; cidx += blockDim.x) amax_merge(best, bi, row[cidx], cidx);
+    if ((v & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0) {   // 16-byte aligned rows: four columns per load
+        const float4* row4 = reinterpret_cast<const float4*>(row);
+#pragma unroll 4
+        for (int q = threadIdx.x; q < (v >> 2); q += blockDim.x) {
+            const float4 w = __ldcs(row4 + q);
+            amax_merge(best, bi, w.x, 4 * q);
+            amax_merge(best, bi, w.y, 4 * q + 1);
+            amax_merge(best, bi, w.z, 4 * q + 2);
+            amax_merge(best, bi, w.w, 4 * q + 3);
+        }
+    } else {
+        for (int cidx = threadIdx.x; cidx < v; cidx += blockDim.x) amax_merge(best, bi, row[cidx], cidx);
+    }
     for (int o = 16; o > 0; o >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, best, o);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
@@ -275,7 +400,7 @@ __global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __res
 }
 
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out) {
-    k_argmax<<<n, 512, 0, c->cur>>>(logits, v, out);
+    k_argmax<<<n, 1024, 0, c->cur>>>(logits, v, out);
     c->launches++;
 }
 
