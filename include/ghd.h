@@ -55,7 +55,9 @@ typedef enum ghd_option {
     GHD_OPT_GRAPH = 3,        /* ghd_verify_step: 0/1 = launch kernels directly, 2 = replay a
                                  CUDA graph captured on first use for the same arguments    */
     GHD_OPT_GEMM_CTAS = 4,    /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
-    GHD_OPT_GEMM_BURST = 5    /* k-steps whose weight loads the tcgen05 GEMM issues together  */
+    GHD_OPT_GEMM_BURST = 5,   /* k-steps whose weight loads the tcgen05 GEMM issues together  */
+    GHD_OPT_NO_PDL = 6        /* 1 = launch every kernel fully serialised (no programmatic
+                                 dependent launch overlap between consecutive kernels)        */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary

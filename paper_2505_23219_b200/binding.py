@@ -19,12 +19,12 @@ __all__ = [
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
     "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
-OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST = 0, 1, 2, 3, 4, 5
+OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
 

@@ -109,6 +109,8 @@ k_attn_simt(const T* __restrict__ q, const T* __restrict__ kc, const T* __restri
 template <typename T>
 __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml, T* __restrict__ out,
                                int splits, int heads, int dh, int max_nodes) {
+    pdl_wait();
+    pdl_trigger();
     const int i = blockIdx.x, h = blockIdx.y, d = heads * dh;
     float m = -INFINITY;
     for (int s = 0; s < splits; ++s) m = fmaxf(m, part_ml[(((size_t)s * max_nodes + i) * heads + h) * 2]);
@@ -168,12 +170,11 @@ void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n) {
     const ghd_model_cfg& m = c->cfg;
     dim3 cgrid(n, m.n_heads);
     if (m.dtype == GHD_F32)
-        k_attn_combine<float><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (float*)out, splits, m.n_heads,
-                                                              m.d_head, m.max_nodes);
+        launch_k(c, true, k_attn_combine<float>, cgrid, m.d_head, 0, (const float*)c->att_o, (const float*)c->att_ml, (float*)out,
+                 splits, m.n_heads, m.d_head, m.max_nodes);
     else
-        k_attn_combine<__half><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (__half*)out, splits, m.n_heads,
-                                                               m.d_head, m.max_nodes);
-    c->launches++;
+        launch_k(c, true, k_attn_combine<__half>, cgrid, m.d_head, 0, (const float*)c->att_o, (const float*)c->att_ml, (__half*)out,
+                 splits, m.n_heads, m.d_head, m.max_nodes);
 }
 
 // ---------------------------------------------------------------------------

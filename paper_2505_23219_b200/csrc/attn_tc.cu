@@ -106,6 +106,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();              // q, the new K/V rows and the mask come from earlier kernels
+    if (threadIdx.x == 0) pdl_trigger();
     // which 64-node groups does any query row of this CTA see?
     if (threadIdx.x >= 64) {
         const int row = row0 + (int)threadIdx.x - 64;
@@ -384,9 +386,8 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         }
         attr_set = true;
     }
-    if (dh == 64) k_attn_tc<64><<<grid, THREADS, attn_smem_bytes<64>(), c->cur>>>(tm_q, tm_k, tm_v, p);
-    else k_attn_tc<128><<<grid, THREADS, attn_smem_bytes<128>(), c->cur>>>(tm_q, tm_k, tm_v, p);
-    c->launches++;
+    if (dh == 64) launch_k(c, true, k_attn_tc<64>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
+    else launch_k(c, true, k_attn_tc<128>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
     launch_attn_combine(c, out, splits, n);
     return GHD_OK;
 }

@@ -197,6 +197,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
+    if (threadIdx.x == 0) pdl_trigger();       // this CTA now owns its shared and tensor memory
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -211,6 +212,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             // thread more cycles than the loads it issues
             int tile = (int)(it_beg / p.kiters), kk = (int)(it_beg - (long long)tile * p.kiters);
             const int my_iters = (int)(it_end - it_beg);
+            const int prefill = my_iters < p.stages ? my_iters : p.stages;   // iterations issued without waiting for a free slot
+            const int kk0 = kk;
             int burst_left = 0;
             for (int i = 0; i < my_iters && ok; ++i) {
                 if (burst_left == 0) {
@@ -233,7 +236,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 } else {
                     tma_load_2d(a_dst, &tm_w, kk * TILE_K, tile * TILE_M, full, pol_stream);
                 }
-                tma_load_2d(b_dst, &tm_x, kk * TILE_K, 0, full, pol_keep);
+                if (i < prefill) {
+                    // weights never change: the first ring-full of weight tiles streams in while the
+                    // previous kernel is still finishing; the activations follow after the wait
+                    if (i == prefill - 1) {
+                        pdl_wait();
+                        for (int q = 0; q < prefill; ++q)
+                            tma_load_2d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, (kk0 + q) % p.kiters * TILE_K, 0,
+                                        smem_u32(&sm->full[q]), pol_keep);
+                    }
+                } else {
+                    tma_load_2d(b_dst, &tm_x, kk * TILE_K, 0, full, pol_keep);
+                }
                 ++issued;
                 if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                 if (++kk == p.kiters) { kk = 0; ++tile; }
@@ -293,6 +307,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int et = threadIdx.x - 64;                       // 0..127 among epilogue threads
+        pdl_wait();                                            // outputs, residual and partial buffers belong to earlier kernels until now
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
         long long it = it_beg;
@@ -461,8 +476,7 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
         c->pending.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
         c->pending.m = m;
     }
-    k_gemm_tc<<<ctas, THREADS, smem, c->cur>>>(tm_w, tm_x, p);
-    c->launches++;
+    launch_k(c, true, k_gemm_tc, ctas, THREADS, smem, tm_w, tm_x, p);
     return GHD_OK;
 }
 

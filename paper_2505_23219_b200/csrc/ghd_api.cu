@@ -161,7 +161,7 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
@@ -209,6 +209,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_ATTN_PATH: if (value > 2) return GHD_EINVAL; c->opt_attn_path = value; break;
         case GHD_OPT_GRAPH: if (value > 2) return GHD_EINVAL; c->opt_graph = value; break;
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
+        case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
         default: return GHD_EINVAL;
     }
@@ -306,7 +307,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
     key.push_back(((uint64_t)(uint32_t)c->opt_gemm_path << 48) | ((uint64_t)(uint32_t)c->opt_attn_splits << 32) |
-                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | ((uint32_t)c->opt_gemm_ctas & 0xfff) | ((uint32_t)c->opt_gemm_burst << 12));
+                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | ((uint32_t)c->opt_gemm_ctas & 0xfff) | ((uint32_t)c->opt_gemm_burst << 12) | ((uint32_t)c->opt_no_pdl << 15));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
         push(lw.wqkv); push(lw.wo); push(lw.w_gate_up); push(lw.w_down); push(lw.rms1); push(lw.rms2);

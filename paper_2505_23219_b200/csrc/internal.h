@@ -7,6 +7,7 @@
 
 #include <map>
 #include <tuple>
+#include <utility>
 #include <vector>
 
 #include "ghd.h"
@@ -63,7 +64,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -89,6 +90,31 @@ struct ghd_ctx {
 };
 
 namespace ghd {
+
+// Programmatic dependent launch.  A kernel launched with `pdl` may start while its predecessor in
+// the stream is still running; it must call pdl_wait() before it touches anything another kernel
+// writes or reads-then-overwrites (only constant weights and its own on-chip set-up may come
+// earlier), and calls pdl_trigger() once its blocks hold the resources later kernels could compete for.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(ghd_ctx* c, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->cur;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pdl && !c->opt_no_pdl) ? 1 : 0;
+    c->launches++;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 size_t carve_workspace(ghd_ctx* c, char* base);   // returns bytes needed; assigns pointers when base != nullptr
 

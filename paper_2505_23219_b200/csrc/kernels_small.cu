@@ -102,6 +102,8 @@ __global__ void k_store_x(const float* __restrict__ xres, T* __restrict__ x, siz
 
 template <typename T>
 __global__ void k_embed(const T* __restrict__ table, const int32_t* __restrict__ tokens, float* __restrict__ xres, int d) {
+    pdl_wait();
+    pdl_trigger();
     const T* row = table + (size_t)tokens[blockIdx.x] * d;
     for (int cidx = threadIdx.x; cidx < d; cidx += blockDim.x) xres[(size_t)blockIdx.x * d + cidx] = to_f32<T>(row[cidx]);
 }
@@ -128,9 +130,8 @@ void launch_store_x(ghd_ctx* c, void* x_out, int n) {
 }
 
 void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n) {
-    GHD_DISPATCH_T(c, (k_embed<float><<<n, 256, 0, c->cur>>>((const float*)embed, tokens, c->xres, c->cfg.d_model)),
-                   (k_embed<__half><<<n, 256, 0, c->cur>>>((const __half*)embed, tokens, c->xres, c->cfg.d_model)));
-    c->launches++;
+    GHD_DISPATCH_T(c, launch_k(c, true, k_embed<float>, n, 256, 0, (const float*)embed, tokens, c->xres, c->cfg.d_model),
+                   launch_k(c, true, k_embed<__half>, n, 256, 0, (const __half*)embed, tokens, c->xres, c->cfg.d_model));
 }
 
 // ---------------------------------------------------------------- RMSNorm
@@ -177,6 +178,8 @@ template <> __device__ __forceinline__ float4 load4<__half>(const __half* p) {
 template <typename T>
 __global__ void k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, T* __restrict__ out, int d, float eps) {
     __shared__ float red[32];
+    pdl_wait();
+    pdl_trigger();
     const float* row = x + (size_t)blockIdx.x * d;
     const int nv = d >> 2;                        // d is a multiple of 8
     float4 v[RMS_V];
@@ -213,9 +216,8 @@ void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out)
     const int d = c->cfg.d_model;
     int threads = ((d / 4 + 31) / 32) * 32;
     if (threads > 1024) threads = 1024;
-    GHD_DISPATCH_T(c, (k_rmsnorm<float><<<n, threads, 0, c->cur>>>(x, (const float*)g, (float*)out, d, c->cfg.rms_eps)),
-                   (k_rmsnorm<__half><<<n, threads, 0, c->cur>>>(x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps)));
-    c->launches++;
+    GHD_DISPATCH_T(c, launch_k(c, true, k_rmsnorm<float>, n, threads, 0, x, (const float*)g, (float*)out, d, c->cfg.rms_eps),
+                   launch_k(c, true, k_rmsnorm<__half>, n, threads, 0, x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps));
 }
 
 // Folds the partial tiles of a deferred-reduction projection into the residual stream and,
@@ -226,6 +228,8 @@ template <typename T>
 __global__ void k_fold_pending(float* __restrict__ xres, const float* __restrict__ part, PendingPartials pp,
                                const T* __restrict__ g, T* __restrict__ h_out, T* __restrict__ x_out, int d, float eps) {
     __shared__ float red[32];
+    pdl_wait();
+    pdl_trigger();
     const int node = blockIdx.x;
     const int nv = d >> 2;
     float4 v[RMS_V];
@@ -278,10 +282,9 @@ void launch_fold_pending(ghd_ctx* c, int n, const void* g, void* h_out, void* x_
     const int d = c->cfg.d_model;
     int threads = (((d / 4 + RMS_V - 1) / RMS_V + 31) / 32) * 32;      // d/4 float4 per row, up to RMS_V per thread
     if (d / 4 <= 1024) threads = ((d / 4 + 31) / 32) * 32;
-    k_fold_pending<__half><<<n, threads, 0, c->cur>>>(c->xres, c->gemm_part, c->pending, (const __half*)g, (__half*)h_out,
-                                                      (__half*)x_out, d, c->cfg.rms_eps);
+    launch_k(c, true, k_fold_pending<__half>, n, threads, 0, c->xres, (const float*)c->gemm_part, c->pending, (const __half*)g,
+             (__half*)h_out, (__half*)x_out, d, c->cfg.rms_eps);
     c->pending.active = 0;
-    c->launches++;
 }
 
 // ---------------------------------------------------------------- RoPE + KV append (un-fused path)
@@ -362,6 +365,8 @@ __device__ __forceinline__ void amax_merge(float& v, int& i, float ov, int oi) {
 __global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __restrict__ out) {
     __shared__ float sv[32];
     __shared__ int si[32];
+    pdl_wait();
+    pdl_trigger();
     const float* row = logits + (size_t)blockIdx.x * v;
     float best = -INFINITY;
     int bi = 0x7fffffff;
@@ -400,8 +405,7 @@ __global__ void k_argmax(const float* __restrict__ logits, int v, int32_t* __res
 }
 
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out) {
-    k_argmax<<<n, 1024, 0, c->cur>>>(logits, v, out);
-    c->launches++;
+    launch_k(c, true, k_argmax, n, 1024, 0, logits, v, out);
 }
 
 // ---------------------------------------------------------------- acceptance
