@@ -129,6 +129,37 @@ __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __
     }
 }
 
+// Same merge, one block per node and four consecutive features per thread (16-byte loads):
+// used when the row width is a multiple of 4, i.e. always for the supported head sizes.
+template <typename T>
+__global__ void k_attn_combine_rows(const float* __restrict__ part_o, const float* __restrict__ part_ml, T* __restrict__ out,
+                                    int splits, int heads, int dh, int max_nodes) {
+    pdl_wait();
+    pdl_trigger();
+    const int i = blockIdx.x, d = heads * dh;
+    for (int f = 4 * threadIdx.x; f < d; f += 4 * blockDim.x) {
+        const int h = f / dh;
+        float ms[16], m = -INFINITY;
+        for (int s = 0; s < splits; ++s) {
+            ms[s] = part_ml[(((size_t)s * max_nodes + i) * heads + h) * 2];
+            m = fmaxf(m, ms[s]);
+        }
+        float den = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < splits; ++s) {
+            if (ms[s] == -INFINITY) continue;
+            const float w = expf(ms[s] - m);
+            den += part_ml[(((size_t)s * max_nodes + i) * heads + h) * 2 + 1] * w;
+            const float4 o = *reinterpret_cast<const float4*>(part_o + ((size_t)s * max_nodes + i) * d + f);
+            acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+        }
+        const float inv = 1.f / den;
+        T* dst = out + (size_t)i * d + f;
+        dst[0] = st_cvt<T>(acc.x * inv); dst[1] = st_cvt<T>(acc.y * inv);
+        dst[2] = st_cvt<T>(acc.z * inv); dst[3] = st_cvt<T>(acc.w * inv);
+    }
+}
+
 }  // namespace
 
 int attn_auto_splits(const ghd_ctx* c, int n, int kv_total) {
@@ -168,6 +199,17 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
 
 void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n) {
     const ghd_model_cfg& m = c->cfg;
+    if (splits <= 16) {
+        int threads = ((m.d_model / 4 + 31) / 32) * 32;
+        if (threads > 1024) threads = 1024;
+        if (m.dtype == GHD_F32)
+            launch_k(c, true, k_attn_combine_rows<float>, n, threads, 0, (const float*)c->att_o, (const float*)c->att_ml,
+                     (float*)out, splits, m.n_heads, m.d_head, m.max_nodes);
+        else
+            launch_k(c, true, k_attn_combine_rows<__half>, n, threads, 0, (const float*)c->att_o, (const float*)c->att_ml,
+                     (__half*)out, splits, m.n_heads, m.d_head, m.max_nodes);
+        return;
+    }
     dim3 cgrid(n, m.n_heads);
     if (m.dtype == GHD_F32)
         launch_k(c, true, k_attn_combine<float>, cgrid, m.d_head, 0, (const float*)c->att_o, (const float*)c->att_ml, (float*)out,

@@ -57,6 +57,12 @@ struct AttnSmem {
     int abort_flag;
 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -83,6 +89,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     const int split = blockIdx.x, h = blockIdx.y, mtile = blockIdx.z;
     const int row0 = mtile * QM;
 
+    if (threadIdx.x == 32) {        // descriptor fetches overlap the barrier set-up
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+    }
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&sm->q_full), 1);
         for (int s = 0; s < KV_STAGES; ++s) { mbar_init(smem_u32(&sm->kv_full[s]), 1); mbar_init(smem_u32(&sm->kv_empty[s]), 1); }
@@ -234,25 +245,35 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const int r = quad * 32 + lane;                        // row inside the tile = tensor-memory lane
         const int row = row0 + r;
         const bool live = row < p.n;
+        const bool warp_live = row0 + quad * 32 < p.n;         // warps whose 32 rows are all padding skip the math
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-        const float c_log2e = 1.4426950408889634f;
+        const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain: s * scale * log2(e)
         float m = -INFINITY, l = 0.f, corr_prev = 1.f;
         float o[DH];
 #pragma unroll
         for (int c = 0; c < DH; ++c) o[c] = 0.f;
+        if (!warp_live) {                                      // padding rows contribute zero rows of P, written once
+#pragma unroll
+            for (int bb = 0; bb < 2; ++bb)
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(p_ptr + bb * P_BYTES + r * 128 + (ch << 4)) = make_uint4(0, 0, 0, 0);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
 
         auto fold_pv = [&](int i, float corr) {
             const int b = i & 1;
             mbar_wait(smem_u32(&sm->pv_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
-            tc_fence_after();
+            if (warp_live) {
+                tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < DH; c0 += 32) {
-                float v[32];
-                tc_ld32(tmem_base + TMEM_PV + b * DH + c0 + lane_off, v);
+                for (int c0 = 0; c0 < DH; c0 += 32) {
+                    float v[32];
+                    tc_ld32(tmem_base + TMEM_PV + b * DH + c0 + lane_off, v);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                    for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                }
+                tc_fence_before();
             }
-            tc_fence_before();
             mbar_arrive(smem_u32(&sm->pv_empty[b]));
         };
 
@@ -269,6 +290,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 }
             }
             mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            if (!warp_live) {
+                mbar_arrive(smem_u32(&sm->s_empty[b]));
+                if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+                mbar_arrive(smem_u32(&sm->p_full[b]));
+                if (i >= 1) fold_pv(i - 1, 1.f);
+                continue;
+            }
             tc_fence_after();
             float s[BN];
             {
@@ -282,36 +310,42 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&sm->s_empty[b]));
-            float tmax = -INFINITY;
+            // hidden keys become -inf once; exp2(-inf) = 0 then needs no further selects
+            if (vis != ~0ull) {
 #pragma unroll
-            for (int j = 0; j < BN; ++j) {
-                s[j] *= p.scale;
-                if ((vis >> j) & 1ull) tmax = fmaxf(tmax, s[j]);
+                for (int j = 0; j < BN; ++j) s[j] = ((vis >> j) & 1ull) ? s[j] : -INFINITY;
             }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < BN; j += 4) {
+                mx[0] = fmaxf(mx[0], s[j]); mx[1] = fmaxf(mx[1], s[j + 1]);
+                mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
+            }
+            const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;
             const float m_new = fmaxf(m, tmax);
-            float corr = 1.f, psum = 0.f;
-            const float mb = (m_new == -INFINITY) ? 0.f : m_new * c_log2e;
-            if (m_new != -INFINITY) corr = (m == -INFINITY) ? 0.f : exp2f(m * c_log2e - mb);
+            const float neg = (m_new == -INFINITY) ? 0.f : -m_new;
+            const float corr = (m_new == -INFINITY) ? 1.f : ex2_approx(m + neg);      // m = -inf gives 0
             // P row -> shared memory, K-major with the 128-byte swizzle the MMA descriptor expects
             if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
             uint8_t* prow = p_ptr + b * P_BYTES + r * 128;
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
                 uint32_t packed[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int j = ch * 8 + 2 * e;
-                    const float p0 = ((vis >> j) & 1ull) ? exp2f(fmaf(s[j], c_log2e, -mb)) : 0.f;
-                    const float p1 = ((vis >> (j + 1)) & 1ull) ? exp2f(fmaf(s[j + 1], c_log2e, -mb)) : 0.f;
+                    const float p0 = ex2_approx(fmaf(s[j], sl2, neg));
+                    const float p1 = ex2_approx(fmaf(s[j + 1], sl2, neg));
+                    ps[e] += p0 + p1;
                     const __half2 hh = __floats2half2_rn(p0, p1);
-                    psum += __low2float(hh) + __high2float(hh);
                     packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
                 }
                 *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(smem_u32(&sm->p_full[b]));
-            l = l * corr + psum;
+            l = l * corr + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
             m = m_new;
             if (i >= 1) fold_pv(i - 1, corr_prev);
             corr_prev = corr;
@@ -322,7 +356,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
             for (int c = 0; c < DH; c += 4) *reinterpret_cast<float4*>(po + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
             float* pm = p.part_ml + (((size_t)split * p.max_nodes + row) * p.heads + h) * 2;
-            pm[0] = m;
+            pm[0] = m * 0.6931471805599453f;                   // back to the natural-log domain the merge kernel uses
             pm[1] = l;
         }
     }

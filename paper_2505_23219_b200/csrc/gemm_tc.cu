@@ -180,6 +180,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     uint32_t tmem_cols = 32;
     while (tmem_cols < 2u * buf_cols) tmem_cols <<= 1;
 
+    if (threadIdx.x == 32) {        // descriptor fetches overlap the barrier set-up
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&sm->full[s]), 1); mbar_init(smem_u32(&sm->empty[s]), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), 4); }
