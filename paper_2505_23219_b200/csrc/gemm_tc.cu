@@ -98,22 +98,25 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
         return;
     }
     if (e.mode == EPI_SWIGLU) {
-        // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows
+        // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows.
+        // After the exchange every thread finishes 16 nodes of one feature: thread `row` takes feature
+        // row & 63 and nodes 16 * (row >> 6) ...  Inputs are gathered first, stores come last (a store
+        // between two loads would serialise them: the compiler cannot prove the pointers distinct).
 #pragma unroll
         for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
         epi_bar();
-        if (row < 64) {
-            const int f = tile * 64 + row;
-            __half* u = (__half*)e.out_t;
+        const int f = row & 63, jb = (row >> 6) * 16;
+        float g[16], up[16];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int node = c0 + j;
-                if (node < p.n) {
-                    const float g = v[j], up = sm->stage_x[j][row + 64];
-                    u[(size_t)node * p.swiglu_f + f] = __float2half_rn(g / (1.f + __expf(-g)) * up);
-                }
-            }
-        }
+        for (int j = 0; j < 16; ++j) { g[j] = sm->stage_x[jb + j][f]; up[j] = sm->stage_x[jb + j][f + 64]; }
+        __half res[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j)      // SiLU(g) * up = g * up / (1 + 2^(-g log2 e))
+            res[j] = __float2half_rn(__fdividef(g[j] * up[j], 1.f + exp2f(-1.4426950408889634f * g[j])));
+        __half* u = (__half*)e.out_t + (size_t)(c0 + jb) * p.swiglu_f + tile * 64 + f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (c0 + jb + j < p.n) u[(size_t)j * p.swiglu_f] = res[j];
         epi_bar();
         return;
     }
@@ -123,30 +126,26 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
     const int section = f / d, el = f - section * d;
     const int head = el / dh, idx = el - head * dh;
     if (section < 2) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
-        epi_bar();
         const int prow = (idx < half) ? row + half : row - half;
         const int t = (idx < half) ? idx : idx - half;
         const float sign = (idx < half) ? -1.f : 1.f;
+        // the table loads go out first so that their latency overlaps the exchange through shared memory
         float2 cs[32];
+        const float2* tab = reinterpret_cast<const float2*>(e.rope + (size_t)c0 * dh + 2 * t);
 #pragma unroll
-        for (int j = 0; j < 32; ++j)       // table loads before any store (see above)
-            cs[j] = (c0 + j < p.n) ? __ldg(reinterpret_cast<const float2*>(e.rope + (size_t)(c0 + j) * dh + 2 * t)) : make_float2(1.f, 0.f);
-        float r[32];
+        for (int j = 0; j < 32; ++j) cs[j] = (c0 + j < p.n) ? __ldg(tab + (size_t)j * half) : make_float2(1.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
-        if (section == 0) {
-            __half* qo = (__half*)e.out_t + (size_t)c0 * d + el;
+        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
+        epi_bar();
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (c0 + j < p.n) qo[(size_t)j * d] = __float2half_rn(r[j]);
-        } else {
-            __half* ko = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx;
+        for (int j = 0; j < 32; ++j) v[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
+        __half* dst;
+        size_t pitch;
+        if (section == 0) { dst = (__half*)e.out_t + (size_t)c0 * d + el; pitch = (size_t)d; }
+        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx; pitch = (size_t)dh; }
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (c0 + j < p.n) ko[(size_t)j * dh] = __float2half_rn(r[j]);
-        }
+        for (int j = 0; j < 32; ++j)
+            if (c0 + j < p.n) dst[(size_t)j * pitch] = __float2half_rn(v[j]);
         epi_bar();
     } else {
 #pragma unroll
@@ -216,7 +215,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             // thread more cycles than the loads it issues
             int tile = (int)(it_beg / p.kiters), kk = (int)(it_beg - (long long)tile * p.kiters);
             const int my_iters = (int)(it_end - it_beg);
-            const int prefill = my_iters < p.stages ? my_iters : p.stages;   // iterations issued without waiting for a free slot
+            const int prefill = my_iters < p.stages / 2 ? my_iters : p.stages / 2;   // weight tiles issued ahead of the dependency wait
             const int kk0 = kk;
             int burst_left = 0;
             for (int i = 0; i < my_iters && ok; ++i) {
@@ -341,39 +340,53 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 // its only unit of this tile), slot 1 when it is the head part of the CTA's last tile
                 const int slot = (it == it_beg) ? 0 : 1;
                 float* mine = p.part + ((size_t)cta * 2 + slot) * slot_elems;
-                for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
-                    float v[32];
-                    tc_ld32(t_addr + c0, v);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
-                if (p.epi.mode == EPI_DEFER) {                 // the consumer kernel sums the partial tiles
-                    if (++buf == 2) { buf = 0; buf_phase ^= 1; }
-                    it += (k1 - k0);
-                    continue;
-                }
-                __threadfence();
-                epi_bar();
                 const long long t_first = (long long)tile * p.kiters;
                 const int c_first = cta_of_iter(t_first, total, G), c_last = cta_of_iter(t_first + p.kiters - 1, total, G);
-                if (et == 0) {
-                    const int old = atomicAdd(p.counters + tile, 1);
-                    sm->last_flag = (old == c_last - c_first) ? 1 : 0;
+                bool finish = false;       // this CTA completes the tile
+                bool dumped = false;
+                if (p.epi.mode != EPI_DEFER) {
+                    // Usually the other contributors handled their share of this tile as the first unit of
+                    // their range, long ago: if all of them have arrived, finish the tile straight from
+                    // tensor memory without the store / fence / count round trips.
+                    if (et == 0) sm->last_flag = (ld_acquire_gpu(p.counters + tile) == c_last - c_first) ? 1 : 0;
+                    epi_bar();
+                    finish = sm->last_flag != 0;
+                    epi_bar();
                 }
-                epi_bar();
-                const bool last = sm->last_flag != 0;
-                epi_bar();
-                if (last) {
-                    __threadfence();
-                    for (int c0 = 0; c0 < p.nb && c0 < p.n; c0 += EPI_CHUNK) {
+                if (!finish) {
+                    for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
                         float v[32];
+                        tc_ld32(t_addr + c0, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
+                    }
+                    dumped = true;
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+                    if (p.epi.mode != EPI_DEFER) {
+                        // count this arrival: the barrier orders every thread's stores before thread 0's
+                        // release, and the release is cumulative over them
+                        epi_bar();
+                        if (et == 0) sm->last_flag = (atom_add_acq_rel_gpu(p.counters + tile, 1) == c_last - c_first) ? 1 : 0;
+                        epi_bar();
+                        finish = sm->last_flag != 0;
+                        epi_bar();
+                    }
+                }
+                if (finish) {
+                    for (int c0 = 0; c0 < p.nb && c0 < p.n; c0 += EPI_CHUNK) {
+                        float v[32], own[32];
+                        if (!dumped) tc_ld32(t_addr + c0, own);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                        // contributors in CTA order; each one's 32 loads are issued together
+                        // contributors in CTA order (fixed order -> reproducible); each one's 32 loads go out together
                         for (int c = c_first; c <= c_last; ++c) {
+                            if (c == cta && !dumped) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] += own[j];
+                                continue;
+                            }
                             const long long cb = total * c / G;
                             const int cslot = (cb >= t_first) ? 0 : 1;
                             const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems + (size_t)c0 * TILE_M + row;
@@ -384,6 +397,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                             for (int j = 0; j < 32; ++j) v[j] += t[j];
                         }
                         epilogue_chunk(p, sm, tile, row, c0, v);
+                    }
+                    if (!dumped) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
                     }
                     if (et == 0) p.counters[tile] = 0;         // ready for the next launch
                 }

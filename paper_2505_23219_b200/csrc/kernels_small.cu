@@ -176,7 +176,7 @@ template <> __device__ __forceinline__ float4 load4<__half>(const __half* p) {
 }
 
 template <typename T>
-__global__ void k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, T* __restrict__ out, int d, float eps) {
+__global__ void __launch_bounds__(1024) k_rmsnorm(const float* __restrict__ x, const T* __restrict__ g, T* __restrict__ out, int d, float eps) {
     __shared__ float red[32];
     pdl_wait();
     pdl_trigger();
@@ -225,7 +225,7 @@ void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out)
 // consecutive features (all inside one 128-row tile), adds that tile's contributors in CTA
 // order (fixed order -> reproducible), then the row's mean square is reduced across the block.
 template <typename T>
-__global__ void k_fold_pending(float* __restrict__ xres, const float* __restrict__ part, PendingPartials pp,
+__global__ void __launch_bounds__(1024) k_fold_pending(float* __restrict__ xres, const float* __restrict__ part, PendingPartials pp,
                                const T* __restrict__ g, T* __restrict__ h_out, T* __restrict__ x_out, int d, float eps) {
     __shared__ float red[32];
     pdl_wait();
@@ -244,11 +244,20 @@ __global__ void k_fold_pending(float* __restrict__ xres, const float* __restrict
             const int c_first = (int)(((t_first + 1) * pp.ctas + pp.total - 1) / pp.total) - 1;
             const int c_last = (int)(((t_first + pp.kiters) * pp.ctas + pp.total - 1) / pp.total) - 1;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c = c_first; c <= c_last; ++c) {
-                const int slot = (pp.total * c / pp.ctas >= t_first) ? 0 : 1;
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)c * 2 + slot) * pp.slot_elems +
-                                                                        (size_t)node * 128 + row));
-                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            for (int cb = c_first; cb <= c_last; cb += 8) {          // up to eight loads in flight, summed in CTA order
+                float4 t[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int c = cb + q;
+                    t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (c <= c_last) {
+                        const int slot = (pp.total * c / pp.ctas >= t_first) ? 0 : 1;
+                        t[q] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)c * 2 + slot) * pp.slot_elems +
+                                                                      (size_t)node * 128 + row));
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { acc.x += t[q].x; acc.y += t[q].y; acc.z += t[q].z; acc.w += t[q].w; }
             }
             float4 x = *reinterpret_cast<const float4*>(xres + (size_t)node * d + f);
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
