@@ -42,8 +42,8 @@ constexpr int THREADS = 192;
 
 struct GemmParams {
     int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
-    int n_tiles, kiters, stages;
-    int burst;                       // k-steps whose loads are issued back to back (adjacent 128-byte chunks of the same weight rows)
+    int n_tiles, kiters, stages;     // kiters = k-chunks per tile; a chunk = ks column slabs of 64 = one pipeline stage
+    int ks, kslabs;                  // slabs per stage, slabs per weight row (k / 64)
     int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
     float* part;                     // [ctas][2][nb][128] float partial tiles
     int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
@@ -164,7 +164,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t* tiles = smem_raw + pad;
-    const uint32_t a_bytes = TILE_M * TILE_K * 2, b_bytes = (uint32_t)p.nb * TILE_K * 2;
+    const uint32_t a_slab = TILE_M * TILE_K * 2, b_slab = (uint32_t)p.nb * TILE_K * 2;
+    const uint32_t a_bytes = p.ks * a_slab, b_bytes = p.ks * b_slab;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     Smem* sm = reinterpret_cast<Smem*>(tiles + (size_t)p.stages * stage_bytes);
     const uint32_t tiles_addr = smem_u32(tiles);
@@ -211,49 +212,34 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            // (tile, kk) advance incrementally: a 64-bit division per k-step would cost this single
-            // thread more cycles than the loads it issues
-            int tile = (int)(it_beg / p.kiters), kk = (int)(it_beg - (long long)tile * p.kiters);
+            // (tile, kc) advance incrementally: a 64-bit division per stage would cost this single thread
+            // more cycles than the loads it issues
+            int tile = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)tile * p.kiters);
             const int my_iters = (int)(it_end - it_beg);
-            const int prefill = my_iters < p.stages / 2 ? my_iters : p.stages / 2;   // weight tiles issued ahead of the dependency wait
-            const int kk0 = kk;
-            int burst_left = 0;
+            // weights never change: the first few weight stages stream in while the previous kernel is still
+            // finishing; the activations of those stages follow after the dependency wait
+            const int prefill = my_iters < p.stages / 2 ? my_iters : p.stages / 2;
+            int pre_kc[MAX_STAGES];
             for (int i = 0; i < my_iters && ok; ++i) {
-                if (burst_left == 0) {
-                    // free the ring slots of a whole burst first, then issue its loads together
-                    uint32_t s2 = stage, ph2 = phase;
-                    for (int j = 0; j < p.burst && i + j < my_iters && ok; ++j) {
-                        if (issued + j >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[s2]), ph2 ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
-                        if (++s2 == (uint32_t)p.stages) { s2 = 0; ph2 ^= 1; }
-                    }
-                    burst_left = p.burst;
-                }
-                --burst_left;
+                if (issued >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
                 if (!ok) break;
                 const uint32_t full = smem_u32(&sm->full[stage]);
                 const uint32_t a_dst = tiles_addr + stage * stage_bytes, b_dst = a_dst + a_bytes;
                 mbar_expect_tx(full, stage_bytes);
-                if (p.swiglu_f) {
-                    tma_load_2d(a_dst, &tm_w, kk * TILE_K, tile * 64, full, pol_stream);
-                    tma_load_2d(a_dst + a_bytes / 2, &tm_w, kk * TILE_K, p.swiglu_f + tile * 64, full, pol_stream);
-                } else {
-                    tma_load_2d(a_dst, &tm_w, kk * TILE_K, tile * TILE_M, full, pol_stream);
-                }
+                tma_load_4d(a_dst, &tm_w, 0, p.swiglu_f ? tile * 64 : tile * TILE_M, 0, kc * p.ks, full, pol_stream);
                 if (i < prefill) {
-                    // weights never change: the first ring-full of weight tiles streams in while the
-                    // previous kernel is still finishing; the activations follow after the wait
+                    pre_kc[i] = kc;
                     if (i == prefill - 1) {
                         pdl_wait();
                         for (int q = 0; q < prefill; ++q)
-                            tma_load_2d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, (kk0 + q) % p.kiters * TILE_K, 0,
-                                        smem_u32(&sm->full[q]), pol_keep);
+                            tma_load_4d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, 0, 0, 0, pre_kc[q] * p.ks, smem_u32(&sm->full[q]), pol_keep);
                     }
                 } else {
-                    tma_load_2d(b_dst, &tm_x, kk * TILE_K, 0, full, pol_keep);
+                    tma_load_4d(b_dst, &tm_x, 0, 0, 0, kc * p.ks, full, pol_keep);
                 }
                 ++issued;
                 if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
-                if (++kk == p.kiters) { kk = 0; ++tile; }
+                if (++kc == p.kiters) { kc = 0; ++tile; }
             }
             if (!ok) {
                 // drain: wait (bounded) until every load issued into the ring has landed
@@ -281,15 +267,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * buf_cols;
-                for (int kk = k0; kk < k1; ++kk) {
+                for (int kc = k0; kc < k1; ++kc) {
                     ok = mbar_wait(smem_u32(&sm->full[stage]), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = tiles_addr + stage * stage_bytes, b_addr = a_addr + a_bytes;
-                    const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(b_addr);
+                    const int nslab = (p.kslabs - kc * p.ks < p.ks) ? p.kslabs - kc * p.ks : p.ks;   // the row's last chunk may be short
+                    for (int sl = 0; sl < nslab; ++sl) {
+                        const uint64_t adesc = smem_desc_sw128(a_addr + sl * a_slab), bdesc = smem_desc_sw128(b_addr + sl * b_slab);
 #pragma unroll
-                    for (int j = 0; j < TILE_K / UMMA_K; ++j)   // +32 bytes along k inside the swizzle row per step
-                        tc_mma_f16(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, (kk > k0 || j > 0) ? 1u : 0u);
+                        for (int j = 0; j < TILE_K / UMMA_K; ++j)   // +32 bytes along k inside the swizzle row per step
+                            tc_mma_f16(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, (kc > k0 || sl > 0 || j > 0) ? 1u : 0u);
+                    }
                     tc_commit(smem_u32(&sm->empty[stage]));    // stage is free once these MMAs have read it
                     if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                 }
@@ -420,29 +409,31 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------- host side
-size_t smem_bytes_for(int nb, int stages) {
-    return 1024 + (size_t)stages * (TILE_M * TILE_K * 2 + (size_t)nb * TILE_K * 2) + sizeof(Smem);
+size_t smem_bytes_for(int nb, int ks, int stages) {
+    return 1024 + (size_t)stages * ks * (TILE_M * TILE_K * 2 + (size_t)nb * TILE_K * 2) + sizeof(Smem);
 }
 
-int pick_stages(int nb) {
+int pick_stages(int nb, int ks) {
     int s = MAX_STAGES;
-    while (s > 2 && smem_bytes_for(nb, s) > 227 * 1024) --s;
+    while (s > 2 && smem_bytes_for(nb, ks, s) > 227 * 1024) --s;
     return s;
 }
 
 }  // namespace
 
 bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
-    if (c->cfg.dtype != GHD_F16 || n < 1 || n > GHD_MAX_NODES || k % 8 || k < TILE_K) return false;
+    if (c->cfg.dtype != GHD_F16 || n < 1 || n > GHD_MAX_NODES || k % TILE_K || k < TILE_K) return false;
     const int n_tiles = (epi_mode == EPI_SWIGLU) ? (m / 2) / 64 : (m + TILE_M - 1) / TILE_M;
     if (n_tiles < 1 || n_tiles > 4096) return false;
     if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
     if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
     if (epi_mode == EPI_DEFER) {
         int ctas = c->opt_gemm_ctas > 0 && c->opt_gemm_ctas < c->sm_count ? c->opt_gemm_ctas : c->sm_count;
-        const long long total = (long long)n_tiles * ((k + TILE_K - 1) / TILE_K);
+        const int ks = (((n + 15) / 16) * 16 <= 128) ? 2 : 1;
+        const int kch = (k / TILE_K + ks - 1) / ks;
+        const long long total = (long long)n_tiles * kch;
         if (ctas > total) ctas = (int)total;
-        if (m % 4 || m > 16384 || total / ctas + 1 > (k + TILE_K - 1) / TILE_K) return false;
+        if (m % 4 || m > 16384 || total / ctas + 1 > kch) return false;
     }
     return true;
 }
@@ -459,17 +450,18 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     p.m = m;
     p.swiglu_f = (epi.mode == EPI_SWIGLU) ? m / 2 : 0;
     p.n_tiles = p.swiglu_f ? p.swiglu_f / 64 : (m + TILE_M - 1) / TILE_M;
-    p.kiters = (k + TILE_K - 1) / TILE_K;
-    p.stages = pick_stages(p.nb);
-    p.burst = c->opt_gemm_burst > 0 ? c->opt_gemm_burst : 1;
-    if (p.burst > p.stages / 2) p.burst = p.stages / 2 > 0 ? p.stages / 2 : 1;
+    p.ks = c->opt_gemm_burst > 0 ? c->opt_gemm_burst : (p.nb <= 128 ? 2 : 1);
+    if (p.ks > 4) p.ks = 4;
+    p.kslabs = k / TILE_K;
+    p.kiters = (p.kslabs + p.ks - 1) / p.ks;
+    p.stages = pick_stages(p.nb, p.ks);
     p.part = c->gemm_part;
     p.counters = c->counters;
     p.status = c->status;
     p.epi = epi;
     CUtensorMap tm_w, tm_x;
-    if (!tmap_rows_x_k(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 64 : TILE_M, &tm_w) ||
-        !tmap_rows_x_k(c, x, (uint64_t)n, (uint64_t)k, (uint32_t)p.nb, &tm_x)) {
+    if (!tmap_slabs(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 2 : 1, p.swiglu_f ? 64 : TILE_M, (uint32_t)p.ks, &tm_w) ||
+        !tmap_slabs(c, x, (uint64_t)n, (uint64_t)k, 1, (uint32_t)p.nb, (uint32_t)p.ks, &tm_x)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: tensor map encoding failed");
         return GHD_ECUDA;
     }
@@ -477,7 +469,7 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     int ctas = c->opt_gemm_ctas > 0 ? c->opt_gemm_ctas : c->sm_count;
     if (ctas > c->sm_count) ctas = c->sm_count;
     if (ctas > total) ctas = (int)total;
-    const size_t smem = smem_bytes_for(p.nb, p.stages);
+    const size_t smem = smem_bytes_for(p.nb, p.ks, p.stages);
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {

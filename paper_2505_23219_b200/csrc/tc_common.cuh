@@ -107,6 +107,13 @@ __device__ __forceinline__ uint32_t instr_desc_f16(int nb, bool b_mn_major = fal
 }
 
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy) : "memory");
+}
+
 __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -132,6 +139,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 bool tmap_rows_x_k(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out);
 // [planes][rows_alloc][cols] of which only the first `rows` rows of each plane are readable
 // (rows beyond read as zero); box = (1 plane x box_rows x 64).
+// Row-major [rows][cols] matrix (cols a multiple of 64) seen as [cols/64][halves][rows/halves][64]:
+// one box = (ks column slabs) x (halves) x (box_rows rows of each half) x 64 elements, which lands in
+// shared memory as ks consecutive [halves*box_rows x 64] swizzled tiles.
+bool tmap_slabs(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t halves, uint32_t box_rows, uint32_t ks,
+                CUtensorMap* out);
 bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
                  uint32_t box_rows, CUtensorMap* out);
 

@@ -129,7 +129,7 @@ def test_linear_cuda_core_path(ghd, shape, n, k, m):
     assert max_rel_err(y.cpu().numpy(), oracle.linear(x, w)) <= 2e-6
 
 
-TC_SHAPES = [(1, 64, 128), (5, 256, 40), (16, 512, 256), (17, 352, 130), (64, 4096, 1024), (64, 11008, 512),
+TC_SHAPES = [(1, 64, 128), (5, 256, 40), (16, 512, 256), (17, 320, 130), (64, 4096, 1024), (64, 11008, 512),
              (100, 1024, 1001), (128, 512, 384), (200, 2048, 256), (256, 1024, 640)]
 
 
