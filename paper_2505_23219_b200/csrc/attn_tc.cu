@@ -4,8 +4,9 @@
 // walked in 64-key units: the cache rows [0, kv_len) first (the dense part: every
 // query sees every row), then the new rows in groups of 64 nodes = one word of the
 // packed ancestor bitmask per query (the sparse part).  A node group whose mask
-// word is zero for every query of the CTA is dropped from the unit list before
-// anything is loaded.  The units are divided evenly among the splits of a head.
+// word is zero for every query of the CTA is dropped before anything of it is
+// loaded.  The cache tiles are divided evenly among the splits of a head and the
+// node groups are dealt to the splits one each.
 //
 // Per unit:  S = Q K^T   (tcgen05.mma, Q and K tile K-major in swizzled shared memory,
 //                         S [128 x 64] float in tensor memory)
@@ -52,6 +53,7 @@ struct AttnSmem {
     uint64_t kv_full[KV_STAGES], kv_empty[KV_STAGES];
     uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2], pv_full[2], pv_empty[2];
     uint64_t drain;
+    uint64_t mask_ready;          // all 128 row threads have merged their mask words into word_or
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
     int abort_flag;
@@ -106,6 +108,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             mbar_init(smem_u32(&sm->pv_empty[b]), 128);
         }
         mbar_init(smem_u32(&sm->drain), 1);
+        mbar_init(smem_u32(&sm->mask_ready), 128);
         for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -119,55 +122,58 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     tc_fence_after();
     pdl_wait();              // q, the new K/V rows and the mask come from earlier kernels
     if (threadIdx.x == 0) pdl_trigger();
-    // which 64-node groups does any query row of this CTA see?
-    if (threadIdx.x >= 64) {
-        const int row = row0 + (int)threadIdx.x - 64;
-        if (row < p.n)
-            for (int w = 0; w < p.n_words; ++w) {
-                const unsigned long long bits = p.mask[(size_t)row * p.n_words + w];
-                if (bits) atomicOr(&sm->word_or[w], bits);
-            }
-    }
-    __syncthreads();
     const uint32_t tmem_base = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
 
-    // unit list: cache tiles, then the visible node groups; this CTA's share of it
+    // Units of this CTA: its share of the cache tiles first (known at once), then the node groups
+    // dealt to this split - group w goes to split (splits - 1 - w mod splits) - that some query
+    // row of the CTA can see.  Which groups are visible is known only after the mask rows have
+    // arrived; every role waits for that (mask_ready) when it reaches the first node group, so
+    // the mask's load latency hides behind the cache tiles.
     const int n_cache = (p.kv_len + BN - 1) / BN;
-    uint32_t act = 0;                                    // bit w set: node group w is visible to some row
+    const int c_beg = n_cache * split / p.splits, c_end = n_cache * (split + 1) / p.splits;
+    uint32_t cand = 0;
 #pragma unroll
     for (int w = 0; w < MAX_UNITS_WORDS; ++w)
-        if (w < p.n_words && sm->word_or[w] != 0ull) act |= 1u << w;
-    const int total = n_cache + __popc(act);
-    const int u_beg = (int)((long long)total * split / p.splits), u_end = (int)((long long)total * (split + 1) / p.splits);
-    const int cnt = u_end - u_beg;
-    auto unit_word = [&](int u) -> int {                 // the (u - n_cache)-th visible node group
-        int left = u - n_cache, w = 0;
+        if (w < p.n_words && p.splits - 1 - (w % p.splits) == split) cand |= 1u << w;
+    // body(i, key0, w): unit number, first key row, node group (-1 for a cache tile); false stops the walk
+    auto walk = [&](auto&& body) -> int {
+        int i = 0;
+        for (int c = c_beg; c < c_end; ++c) {
+            if (!body(i, c * BN, -1)) return i;
+            ++i;
+        }
+        if (cand) {
+            mbar_wait(smem_u32(&sm->mask_ready), 0, abort_flag, p.status, DEV_TIMEOUT_EPI);
 #pragma unroll
-        for (int a = 0; a < MAX_UNITS_WORDS; ++a)
-            if ((act >> a) & 1u) { if (left == 0) w = a; --left; }
-        return w;
+            for (int w = 0; w < MAX_UNITS_WORDS; ++w)
+                if (((cand >> w) & 1u) && sm->word_or[w] != 0ull) {
+                    if (!body(i, p.kv_len + 64 * w, w)) return i;
+                    ++i;
+                }
+        }
+        return i;
     };
-    auto unit_key0 = [&](int u) -> int { return u < n_cache ? u * BN : p.kv_len + 64 * unit_word(u); };
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0 && cnt > 0) {
+        if (lane == 0) {
             uint64_t pol_q, pol_kv;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_q));
             if (gridDim.z > 1) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_kv));
             else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_kv));
-            mbar_expect_tx(smem_u32(&sm->q_full), Q_BYTES);
-#pragma unroll
-            for (int s = 0; s < SLABS; ++s)
-                tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            for (int i = 0; i < cnt; ++i) {
+            walk([&](int i, int key0, int) -> bool {
+                if (i == 0) {
+                    mbar_expect_tx(smem_u32(&sm->q_full), Q_BYTES);
+#pragma unroll
+                    for (int s = 0; s < SLABS; ++s)
+                        tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
+                }
                 if (issued >= KV_STAGES) ok = mbar_wait(smem_u32(&sm->kv_empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
-                if (!ok) break;
-                const int key0 = unit_key0(u_beg + i);
+                if (!ok) return false;
                 const uint32_t full = smem_u32(&sm->kv_full[stage]);
                 const uint32_t k_dst = kv_addr + stage * STAGE_BYTES, v_dst = k_dst + SLABS * KV_SLAB;
                 mbar_expect_tx(full, STAGE_BYTES);
@@ -178,8 +184,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 }
                 ++issued;
                 if (++stage == KV_STAGES) { stage = 0; phase ^= 1; }
-            }
+                return true;
+            });
             if (!ok) {
+                // drain: wait (bounded) for every load issued into the ring, and for Q
                 const int inflight = issued < KV_STAGES ? issued : KV_STAGES;
                 uint32_t s = stage, ph = phase;
                 for (int q = 0; q < inflight; ++q) {
@@ -191,49 +199,55 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        if (lane == 0 && cnt > 0) {
+        if (lane == 0) {
             const uint32_t idesc_s = instr_desc_f16(BN, false);          // S: N = 64 keys, K tile K-major
-            const uint32_t idesc_pv = instr_desc_f16(64, true);          // PV: N = 64 of d_head, V is N-major
-            bool ok = mbar_wait(smem_u32(&sm->q_full), 0, abort_flag, p.status, DEV_TIMEOUT_MMA);
-            tc_fence_after();
+            const uint32_t idesc_pv = instr_desc_f16(DH, true);          // PV: N = d_head, V is N-major
+            // operand descriptors are built once; per MMA only the 16-byte-unit address field moves
+            const uint64_t q_desc = smem_desc_sw128(q_addr), k_desc = smem_desc_sw128(kv_addr);
+            const uint64_t p_desc = smem_desc_sw128(p_addr);
+            // V: rows = keys (the MMA K dimension), 64 d_head columns per 128-byte row, the next 64
+            // columns one slab (KV_SLAB bytes) further: that distance is the leading-dimension offset
+            const uint64_t v_desc = smem_desc_sw128(kv_addr + SLABS * KV_SLAB, KV_SLAB);
+            bool ok = true, have_q = false;
             auto issue_pv = [&](int i) -> bool {
                 const int b = i & 1, stage = i % KV_STAGES;
                 if (!mbar_wait(smem_u32(&sm->p_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) return false;
                 if (i >= 2 && !mbar_wait(smem_u32(&sm->pv_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM)) return false;
                 tc_fence_after();
-                const uint32_t v_addr = kv_addr + stage * STAGE_BYTES + SLABS * KV_SLAB;
-                const uint64_t pdesc = smem_desc_sw128(p_addr + b * P_BYTES);
+                const uint32_t d_tmem = tmem_base + TMEM_PV + b * DH;
+                const uint64_t pd = p_desc + (uint64_t)((b * P_BYTES) >> 4);
+                const uint64_t vd = v_desc + (uint64_t)((stage * STAGE_BYTES) >> 4);
 #pragma unroll
-                for (int s = 0; s < SLABS; ++s) {
-                    const uint32_t d_tmem = tmem_base + TMEM_PV + b * DH + s * 64;
-#pragma unroll
-                    for (int ks = 0; ks < BN / 16; ++ks)     // 16 keys per MMA: +32 B along P's rows, +16 rows of V
-                        tc_mma_f16(d_tmem, pdesc + (uint64_t)(ks * 2), smem_desc_sw128(v_addr + s * KV_SLAB + ks * 16 * 128),
-                                   idesc_pv, ks > 0 ? 1u : 0u);
-                }
+                for (int ks = 0; ks < BN / 16; ++ks)     // 16 keys per MMA: +32 B along P's rows, +16 rows of V
+                    tc_mma_f16(d_tmem, pd + (uint64_t)(ks * 2), vd + (uint64_t)((ks * 16 * 128) >> 4), idesc_pv, ks > 0 ? 1u : 0u);
                 tc_commit(smem_u32(&sm->pv_full[b]));
                 tc_commit(smem_u32(&sm->kv_empty[stage]));
                 tc_commit(smem_u32(&sm->p_empty[b]));
                 return true;
             };
-            for (int i = 0; i < cnt && ok; ++i) {
+            const int cnt = walk([&](int i, int, int) -> bool {
+                if (!have_q) {
+                    ok = mbar_wait(smem_u32(&sm->q_full), 0, abort_flag, p.status, DEV_TIMEOUT_MMA);
+                    have_q = true;
+                }
                 const int b = i & 1, stage = i % KV_STAGES;
-                ok = mbar_wait(smem_u32(&sm->kv_full[stage]), (i / KV_STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA);
+                if (ok) ok = mbar_wait(smem_u32(&sm->kv_full[stage]), (i / KV_STAGES) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA);
                 if (ok && i >= 2) ok = mbar_wait(smem_u32(&sm->s_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM);
-                if (!ok) break;
+                if (!ok) return false;
                 tc_fence_after();
-                const uint32_t k_addr = kv_addr + stage * STAGE_BYTES;
                 const uint32_t d_tmem = tmem_base + TMEM_S + b * BN;
+                const uint64_t kd = k_desc + (uint64_t)((stage * STAGE_BYTES) >> 4);
 #pragma unroll
                 for (int s = 0; s < SLABS; ++s)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        tc_mma_f16(d_tmem, smem_desc_sw128(q_addr + s * Q_SLAB) + (uint64_t)(ks * 2),
-                                   smem_desc_sw128(k_addr + s * KV_SLAB) + (uint64_t)(ks * 2), idesc_s, (s > 0 || ks > 0) ? 1u : 0u);
+                        tc_mma_f16(d_tmem, q_desc + (uint64_t)(((s * Q_SLAB) >> 4) + ks * 2), kd + (uint64_t)(((s * KV_SLAB) >> 4) + ks * 2),
+                                   idesc_s, (s > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&sm->s_full[b]));
                 if (i >= 1) ok = issue_pv(i - 1);
-            }
-            if (ok) ok = issue_pv(cnt - 1);
+                return ok;
+            });
+            if (ok && cnt > 0) ok = issue_pv(cnt - 1);
             if (!ok) {
                 tc_commit(smem_u32(&sm->drain));
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain), 0); ++spin) __nanosleep(64);
@@ -248,6 +262,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const bool warp_live = row0 + quad * 32 < p.n;         // warps whose 32 rows are all padding skip the math
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
         const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain: s * scale * log2(e)
+        // this row's mask words stay in registers; their OR over the CTA's rows tells every role
+        // which node groups exist for this CTA
+        unsigned long long myw[MAX_UNITS_WORDS];
+#pragma unroll
+        for (int w = 0; w < MAX_UNITS_WORDS; ++w) {
+            myw[w] = (live && w < p.n_words) ? p.mask[(size_t)row * p.n_words + w] : 0ull;
+            if (myw[w]) atomicOr(&sm->word_or[w], myw[w]);
+        }
+        mbar_arrive(smem_u32(&sm->mask_ready));
         float m = -INFINITY, l = 0.f, corr_prev = 1.f;
         float o[DH];
 #pragma unroll
@@ -277,17 +300,16 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             mbar_arrive(smem_u32(&sm->pv_empty[b]));
         };
 
-        for (int i = 0; i < cnt; ++i) {
-            const int u = u_beg + i, b = i & 1;
+        const int cnt = walk([&](int i, int key0, int w) -> bool {
+            const int b = i & 1;
             // visibility of the 64 keys of this unit for this row
             unsigned long long vis = 0ull;
-            if (live) {
-                if (u < n_cache) {
-                    const int valid = p.kv_len - u * BN;
-                    vis = valid >= 64 ? ~0ull : ((1ull << valid) - 1ull);
-                } else {
-                    vis = p.mask[(size_t)row * p.n_words + unit_word(u)];
-                }
+            if (w < 0) {
+                const int valid = p.kv_len - key0;
+                if (live) vis = valid >= 64 ? ~0ull : ((1ull << valid) - 1ull);
+            } else {
+#pragma unroll
+                for (int a = 0; a < MAX_UNITS_WORDS; ++a) if (a == w) vis = myw[a];
             }
             mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
             if (!warp_live) {
@@ -295,7 +317,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 mbar_arrive(smem_u32(&sm->p_full[b]));
                 if (i >= 1) fold_pv(i - 1, 1.f);
-                continue;
+                return true;
             }
             tc_fence_after();
             float s[BN];
@@ -349,7 +371,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             m = m_new;
             if (i >= 1) fold_pv(i - 1, corr_prev);
             corr_prev = corr;
-        }
+            return true;
+        });
         if (cnt > 0) fold_pv(cnt - 1, corr_prev);
         if (live) {
             float* po = p.part_o + ((size_t)split * p.max_nodes + row) * (size_t)(p.heads * DH) + h * DH;

@@ -88,12 +88,14 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
     for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
 }
 
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 64
-// halfs (128 B), 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+// Shared-memory matrix descriptor for a 128-byte-swizzled operand made of 128-byte rows, 8-row
+// groups 1024 B apart.  K-major operand: rows = M/N index, the leading offset is unused.
+// N-major operand (rows = K index, 64 N-elements per row): lbo_bytes is the distance to the
+// next 64 N-elements.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes = 16) {
     uint64_t d = 0;
     d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;   // leading byte offset
     d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
     d |= (uint64_t)2 << 61;                           // 128-byte swizzle
