@@ -218,10 +218,12 @@ def run_gpu(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         barrier()
+        torch.cuda.nvtx.range_push("timed")
         ev0.record()
         for _ in range(args.steps):
             step()
         ev1.record()
+        torch.cuda.nvtx.range_pop()
         launches = ghd.ghd_launch_count(ctx) - l0
         barrier()
         ms = ev0.elapsed_time(ev1)
@@ -258,11 +260,13 @@ def run_gpu(args):
         ghd.ghd_linear(ctx, xh, lw.t["w_gate_up"], yraw)
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    torch.cuda.nvtx.range_push("roofline")
     k0.record()
     for _ in range(reps):
         for lw in g_layers:
             ghd.ghd_linear(ctx, xh, lw.t["w_gate_up"], yraw)
     k1.record()
+    torch.cuda.nvtx.range_pop()
     torch.cuda.synchronize()
     ghd.ghd_sync_status(ctx)
     kern_ms = k0.elapsed_time(k1) / (reps * len(g_layers))
