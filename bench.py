@@ -62,6 +62,21 @@ def algorithmic_bytes(shape, n, kv_len):
     return shape.n_layers * per_layer + shape.vocab * d * s + n * d * s + n * shape.vocab * 4
 
 
+# DRAM bytes per launch of the roofline kernel from the ncu capture summarised in
+# profiles/k_gemm_tc_gate_up_projection_llama7b.md; valid only for the kernel source it was taken on.
+NCU_TRAFFIC = {"gemm_tc_sha256_16": "22c0415f88c8eb4f", "bytes_per_launch": 186.5e6}
+
+
+def ncu_traffic():
+    import hashlib
+    src = ROOT / "paper_2505_23219_b200" / "csrc" / "gemm_tc.cu"
+    try:
+        same = hashlib.sha256(src.read_bytes()).hexdigest()[:16] == NCU_TRAFFIC["gemm_tc_sha256_16"]
+    except OSError:
+        same = False
+    return NCU_TRAFFIC["bytes_per_launch"] if same else None
+
+
 def measured_peak():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -301,7 +316,7 @@ def run_gpu(args):
             "roofline": {"bound": "hbm", "kernel": "k_gemm_tc (gate/up projection, [2*11008 x 4096] half, raw float output)",
                          "achieved": kern_bytes / (kern_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                          "frac": kern_bytes / (kern_ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
-                         "us_per_launch": kern_ms * 1e3, "bytes_per_launch": kern_bytes, "traffic": None},
+                         "us_per_launch": kern_ms * 1e3, "bytes_per_launch": kern_bytes, "traffic": ncu_traffic()},
         }
         if world == 1 and not args.no_cpu:
             v, cores, desc = time_oracle_sample(shape, n, kv_len, parent, tokens, min(shape.n_layers, 8))
