@@ -21,7 +21,9 @@
 // softmax aligned by a scaling factor at the end).
 //
 // Warp 0 = TMA producer, warp 1 = MMA issuer + tensor-memory owner, warps 2..5 =
-// softmax (128 threads = 128 tensor-memory lanes).  All waits are bounded.
+// softmax (128 threads = 128 tensor-memory lanes).  All waits are bounded.  Cache tiles that
+// lie wholly below kv_len cannot be touched by the preceding kernel, so the producer requests
+// the first of them before it waits for that kernel to finish.
 #include <cstdio>
 
 #include "internal.h"
@@ -120,7 +122,6 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();              // q, the new K/V rows and the mask come from earlier kernels
     if (threadIdx.x == 0) pdl_trigger();
     const uint32_t tmem_base = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
@@ -162,6 +163,21 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_q));
             if (gridDim.z > 1) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_kv));
             else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_kv));
+            auto load_kv = [&](uint32_t st, int key0) {
+                const uint32_t full = smem_u32(&sm->kv_full[st]);
+                const uint32_t k_dst = kv_addr + st * STAGE_BYTES, v_dst = k_dst + SLABS * KV_SLAB;
+                mbar_expect_tx(full, STAGE_BYTES);
+#pragma unroll
+                for (int s = 0; s < SLABS; ++s) {
+                    tma_load_3d(k_dst + s * KV_SLAB, &tm_k, s * 64, key0, h, full, pol_kv);
+                    tma_load_3d(v_dst + s * KV_SLAB, &tm_v, s * 64, key0, h, full, pol_kv);
+                }
+            };
+            // cache tiles wholly below kv_len are not written by the preceding kernel: request the
+            // first ring-full of them before waiting for that kernel to finish
+            int pre = 0;
+            for (int c = c_beg; c < c_end && pre < KV_STAGES && (c + 1) * BN <= p.kv_len; ++c, ++pre) load_kv(pre, c * BN);
+            pdl_wait();
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
@@ -172,29 +188,26 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     for (int s = 0; s < SLABS; ++s)
                         tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
                 }
-                if (issued >= KV_STAGES) ok = mbar_wait(smem_u32(&sm->kv_empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
-                if (!ok) return false;
-                const uint32_t full = smem_u32(&sm->kv_full[stage]);
-                const uint32_t k_dst = kv_addr + stage * STAGE_BYTES, v_dst = k_dst + SLABS * KV_SLAB;
-                mbar_expect_tx(full, STAGE_BYTES);
-#pragma unroll
-                for (int s = 0; s < SLABS; ++s) {
-                    tma_load_3d(k_dst + s * KV_SLAB, &tm_k, s * 64, key0, h, full, pol_kv);
-                    tma_load_3d(v_dst + s * KV_SLAB, &tm_v, s * 64, key0, h, full, pol_kv);
+                if (i >= pre) {
+                    if (issued >= KV_STAGES) ok = mbar_wait(smem_u32(&sm->kv_empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+                    if (!ok) return false;
+                    load_kv(stage, key0);
                 }
                 ++issued;
                 if (++stage == KV_STAGES) { stage = 0; phase ^= 1; }
                 return true;
             });
             if (!ok) {
-                // drain: wait (bounded) for every load issued into the ring, and for Q
-                const int inflight = issued < KV_STAGES ? issued : KV_STAGES;
-                uint32_t s = stage, ph = phase;
+                // drain: wait (bounded) for every load still in flight, and for Q
+                const int outstanding = issued > pre ? issued : pre;
+                const int inflight = outstanding < KV_STAGES ? outstanding : KV_STAGES;
                 for (int q = 0; q < inflight; ++q) {
-                    if (s == 0) { s = KV_STAGES - 1; ph ^= 1; } else --s;
-                    for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->kv_full[s]), ph); ++spin) __nanosleep(64);
+                    const int idx = outstanding - 1 - q;
+                    for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->kv_full[idx % KV_STAGES]), (idx / KV_STAGES) & 1); ++spin)
+                        __nanosleep(64);
                 }
-                for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->q_full), 0); ++spin) __nanosleep(64);
+                if (issued > 0)
+                    for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->q_full), 0); ++spin) __nanosleep(64);
             }
         }
     } else if (warp == 1) {
@@ -262,6 +275,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const bool warp_live = row0 + quad * 32 < p.n;         // warps whose 32 rows are all padding skip the math
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
         const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain: s * scale * log2(e)
+        pdl_wait();                                            // the mask comes from an earlier kernel
         // this row's mask words stay in registers; their OR over the CTA's rows tells every role
         // which node groups exist for this CTA
         unsigned long long myw[MAX_UNITS_WORDS];
