@@ -20,8 +20,9 @@
 // split; k_attn_combine merges the splits (paper Sec. III-B-2: per-partition
 // softmax aligned by a scaling factor at the end).
 //
-// Warp 0 = TMA producer, warp 1 = MMA issuer + tensor-memory owner, warps 2..5 =
-// softmax (128 threads = 128 tensor-memory lanes).  All waits are bounded.  Cache tiles that
+// Warp 0 = TMA producer, warp 1 = issuer of the S MMAs + tensor-memory owner, warps 2..5 =
+// softmax (128 threads = 128 tensor-memory lanes), warp 6 = issuer of the PV MMAs (two issuing
+// threads because one thread's MMA issue rate, not the tensor pipe, was the limit).  All waits are bounded.  Cache tiles that
 // lie wholly below kv_len cannot be touched by the preceding kernel, so the producer requests
 // the first of them before it waits for that kernel to finish.
 #include <cstdio>
@@ -38,7 +39,7 @@ using namespace tc;
 constexpr int QM = 128;        // query rows per CTA (MMA M)
 constexpr int BN = 64;         // keys per unit (MMA N of S, MMA K of PV)
 constexpr int KV_STAGES = 4;
-constexpr int THREADS = 192;
+constexpr int THREADS = 224;
 constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 
 struct AttnParams {
@@ -54,7 +55,7 @@ struct AttnSmem {
     uint64_t q_full;
     uint64_t kv_full[KV_STAGES], kv_empty[KV_STAGES];
     uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2], pv_full[2], pv_empty[2];
-    uint64_t drain;
+    uint64_t drain, drain_pv;
     uint64_t mask_ready;          // all 128 row threads have merged their mask words into word_or
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
@@ -110,6 +111,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             mbar_init(smem_u32(&sm->pv_empty[b]), 128);
         }
         mbar_init(smem_u32(&sm->drain), 1);
+        mbar_init(smem_u32(&sm->drain_pv), 1);
         mbar_init(smem_u32(&sm->mask_ready), 128);
         for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
         sm->abort_flag = 0;
@@ -211,34 +213,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
+        // ------------------------------------------------ issuer of S = Q K^T
         if (lane == 0) {
             const uint32_t idesc_s = instr_desc_f16(BN, false);          // S: N = 64 keys, K tile K-major
-            const uint32_t idesc_pv = instr_desc_f16(DH, true);          // PV: N = d_head, V is N-major
             // operand descriptors are built once; per MMA only the 16-byte-unit address field moves
             const uint64_t q_desc = smem_desc_sw128(q_addr), k_desc = smem_desc_sw128(kv_addr);
-            const uint64_t p_desc = smem_desc_sw128(p_addr);
-            // V: rows = keys (the MMA K dimension), 64 d_head columns per 128-byte row, the next 64
-            // columns one slab (KV_SLAB bytes) further: that distance is the leading-dimension offset
-            const uint64_t v_desc = smem_desc_sw128(kv_addr + SLABS * KV_SLAB, KV_SLAB);
             bool ok = true, have_q = false;
-            auto issue_pv = [&](int i) -> bool {
-                const int b = i & 1, stage = i % KV_STAGES;
-                if (!mbar_wait(smem_u32(&sm->p_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA)) return false;
-                if (i >= 2 && !mbar_wait(smem_u32(&sm->pv_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM)) return false;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + TMEM_PV + b * DH;
-                const uint64_t pd = p_desc + (uint64_t)((b * P_BYTES) >> 4);
-                const uint64_t vd = v_desc + (uint64_t)((stage * STAGE_BYTES) >> 4);
-#pragma unroll
-                for (int ks = 0; ks < BN / 16; ++ks)     // 16 keys per MMA: +32 B along P's rows, +16 rows of V
-                    tc_mma_f16(d_tmem, pd + (uint64_t)(ks * 2), vd + (uint64_t)((ks * 16 * 128) >> 4), idesc_pv, ks > 0 ? 1u : 0u);
-                tc_commit(smem_u32(&sm->pv_full[b]));
-                tc_commit(smem_u32(&sm->kv_empty[stage]));
-                tc_commit(smem_u32(&sm->p_empty[b]));
-                return true;
-            };
-            const int cnt = walk([&](int i, int, int) -> bool {
+            walk([&](int i, int, int) -> bool {
                 if (!have_q) {
                     ok = mbar_wait(smem_u32(&sm->q_full), 0, abort_flag, p.status, DEV_TIMEOUT_MMA);
                     have_q = true;
@@ -257,13 +238,42 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         tc_mma_f16(d_tmem, q_desc + (uint64_t)(((s * Q_SLAB) >> 4) + ks * 2), kd + (uint64_t)(((s * KV_SLAB) >> 4) + ks * 2),
                                    idesc_s, (s > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&sm->s_full[b]));
-                if (i >= 1) ok = issue_pv(i - 1);
-                return ok;
+                return true;
             });
-            if (ok && cnt > 0) ok = issue_pv(cnt - 1);
             if (!ok) {
                 tc_commit(smem_u32(&sm->drain));
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain), 0); ++spin) __nanosleep(64);
+            }
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------ issuer of PV = P V
+        if (lane == 0) {
+            const uint32_t idesc_pv = instr_desc_f16(DH, true);          // PV: N = d_head, V is N-major
+            const uint64_t p_desc = smem_desc_sw128(p_addr);
+            // V: rows = keys (the MMA K dimension), 64 d_head columns per 128-byte row, the next 64
+            // columns one slab (KV_SLAB bytes) further: that distance is the leading-dimension offset
+            const uint64_t v_desc = smem_desc_sw128(kv_addr + SLABS * KV_SLAB, KV_SLAB);
+            bool ok = true;
+            walk([&](int i, int, int) -> bool {
+                const int b = i & 1, stage = i % KV_STAGES;
+                ok = mbar_wait(smem_u32(&sm->p_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_MMA);
+                if (ok && i >= 2) ok = mbar_wait(smem_u32(&sm->pv_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_TMEM);
+                if (!ok) return false;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + TMEM_PV + b * DH;
+                const uint64_t pd = p_desc + (uint64_t)((b * P_BYTES) >> 4);
+                const uint64_t vd = v_desc + (uint64_t)((stage * STAGE_BYTES) >> 4);
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)     // 16 keys per MMA: +32 B along P's rows, +16 rows of V
+                    tc_mma_f16(d_tmem, pd + (uint64_t)(ks * 2), vd + (uint64_t)((ks * 16 * 128) >> 4), idesc_pv, ks > 0 ? 1u : 0u);
+                tc_commit(smem_u32(&sm->pv_full[b]));
+                tc_commit(smem_u32(&sm->kv_empty[stage]));   // P V is the last reader of the stage (S of the same unit came first)
+                tc_commit(smem_u32(&sm->p_empty[b]));
+                return true;
+            });
+            if (!ok) {
+                tc_commit(smem_u32(&sm->drain_pv));
+                for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain_pv), 0); ++spin) __nanosleep(64);
             }
         }
     } else {
