@@ -60,7 +60,11 @@ struct AttnSmem {
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
     int abort_flag;
+    float xmax[2][QM];            // row-pair mode: the two threads of a row exchange their partial maxima
+    float xl[QM];                 // ... and, at the end, their partial sums
 };
+
+__device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -68,7 +72,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-template <int DH>
+// PAIR: at most 64 query rows.  The queries are loaded twice (tile rows r and r + 64 hold the same
+// query), so S, P and PV come out duplicated and two threads share a row: thread r takes the
+// first 32 keys of a unit and the first half of d_head, thread r + 64 the rest.  This halves the
+// per-unit softmax time, which is what bounds the kernel at small trees.
+template <int DH, bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
@@ -187,8 +195,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 if (i == 0) {
                     mbar_expect_tx(smem_u32(&sm->q_full), Q_BYTES);
 #pragma unroll
-                    for (int s = 0; s < SLABS; ++s)
-                        tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
+                    for (int s = 0; s < SLABS; ++s) {
+                        if constexpr (PAIR) {      // 64-row box, twice: rows 64..127 repeat rows 0..63
+                            tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
+                            tma_load_2d(q_addr + s * Q_SLAB + 64 * 128, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
+                        } else {
+                            tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
+                        }
+                    }
                 }
                 if (i >= pre) {
                     if (issued >= KV_STAGES) ok = mbar_wait(smem_u32(&sm->kv_empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
@@ -274,6 +288,138 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             if (!ok) {
                 tc_commit(smem_u32(&sm->drain_pv));
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain_pv), 0); ++spin) __nanosleep(64);
+            }
+        }
+    } else if constexpr (PAIR) {
+        // ------------------------------------------------ softmax warps, two threads per query row
+        constexpr int HC = BN / 2;                             // keys of a unit per thread
+        constexpr int HD = DH / 2;                             // d_head columns per thread
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                        // tensor-memory lane
+        const int half = r >> 6, row = r & 63;                 // which half of the row's work, query row
+        const bool live = row < p.n;
+        const bool warp_live = (quad & 1) * 32 < p.n;          // warps whose 32 rows are all padding skip the math
+        const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+        const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain
+        pdl_wait();                                            // the mask comes from an earlier kernel
+        unsigned long long myw[MAX_UNITS_WORDS];
+#pragma unroll
+        for (int w = 0; w < MAX_UNITS_WORDS; ++w) {
+            myw[w] = (live && w < p.n_words) ? p.mask[(size_t)row * p.n_words + w] : 0ull;
+            if (myw[w] && half == 0) atomicOr(&sm->word_or[w], myw[w]);
+        }
+        mbar_arrive(smem_u32(&sm->mask_ready));
+        float m = -INFINITY, l = 0.f, corr_prev = 1.f;         // l: sum over this thread's keys only
+        float o[HD];
+#pragma unroll
+        for (int c = 0; c < HD; ++c) o[c] = 0.f;
+        if (!warp_live) {                                      // padding rows contribute zero rows of P, written once
+#pragma unroll
+            for (int bb = 0; bb < 2; ++bb)
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(p_ptr + bb * P_BYTES + r * 128 + (ch << 4)) = make_uint4(0, 0, 0, 0);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+
+        auto fold_pv = [&](int i, float corr) {
+            const int b = i & 1;
+            mbar_wait(smem_u32(&sm->pv_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            if (warp_live) {
+                tc_fence_after();
+#pragma unroll
+                for (int c0 = 0; c0 < HD; c0 += 32) {
+                    float v[32];
+                    tc_ld32(tmem_base + TMEM_PV + b * DH + half * HD + c0 + lane_off, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                }
+                tc_fence_before();
+            }
+            mbar_arrive(smem_u32(&sm->pv_empty[b]));
+        };
+
+        const int cnt = walk([&](int i, int key0, int w) -> bool {
+            const int b = i & 1;
+            // visibility of this thread's 32 keys
+            uint32_t bits = 0u;
+            if (w < 0) {
+                const int valid = p.kv_len - key0 - half * HC;
+                if (live) bits = valid >= HC ? 0xffffffffu : (valid > 0 ? ((1u << valid) - 1u) : 0u);
+            } else {
+#pragma unroll
+                for (int a = 0; a < MAX_UNITS_WORDS; ++a) if (a == w) bits = (uint32_t)(myw[a] >> (half * HC));
+            }
+            mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            if (!warp_live) {
+                mbar_arrive(smem_u32(&sm->s_empty[b]));
+                pair_bar();                                    // every softmax thread takes part in the exchange barrier
+                if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+                mbar_arrive(smem_u32(&sm->p_full[b]));
+                if (i >= 1) fold_pv(i - 1, 1.f);
+                return true;
+            }
+            tc_fence_after();
+            float s[HC];
+            tc_ld32(tmem_base + TMEM_S + b * BN + half * HC + lane_off, s);
+            tc_fence_before();
+            mbar_arrive(smem_u32(&sm->s_empty[b]));
+            if (bits != 0xffffffffu) {
+#pragma unroll
+                for (int j = 0; j < HC; ++j) s[j] = ((bits >> j) & 1u) ? s[j] : -INFINITY;
+            }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < HC; j += 4) {
+                mx[0] = fmaxf(mx[0], s[j]); mx[1] = fmaxf(mx[1], s[j + 1]);
+                mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
+            }
+            const float mine = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            sm->xmax[b][r] = mine;                             // the partner thread (lane r ^ 64) holds the other 32 keys
+            pair_bar();
+            const float tmax = fmaxf(mine, sm->xmax[b][r ^ 64]) * sl2;
+            const float m_new = fmaxf(m, tmax);
+            const float neg = (m_new == -INFINITY) ? 0.f : -m_new;
+            const float corr = (m_new == -INFINITY) ? 1.f : ex2_approx(m + neg);
+            if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
+            // this thread's 32 probabilities go into both copies of the row (tile rows row and row + 64)
+            uint8_t* prow = p_ptr + b * P_BYTES + row * 128;
+            float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t packed[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int j = q * 8 + 2 * e;
+                    const float p0 = ex2_approx(fmaf(s[j], sl2, neg));
+                    const float p1 = ex2_approx(fmaf(s[j + 1], sl2, neg));
+                    ps[e] += p0 + p1;
+                    const __half2 hh = __floats2half2_rn(p0, p1);
+                    packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                const uint32_t off = (uint32_t)(((half * 4 + q) ^ (row & 7)) << 4);
+                const uint4 val = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                *reinterpret_cast<uint4*>(prow + off) = val;
+                *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(smem_u32(&sm->p_full[b]));
+            l = l * corr + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+            m = m_new;
+            if (i >= 1) fold_pv(i - 1, corr_prev);
+            corr_prev = corr;
+            return true;
+        });
+        if (cnt > 0) fold_pv(cnt - 1, corr_prev);
+        sm->xl[r] = l;
+        pair_bar();
+        if (live) {
+            float* po = p.part_o + ((size_t)split * p.max_nodes + row) * (size_t)(p.heads * DH) + h * DH + half * HD;
+#pragma unroll
+            for (int c = 0; c < HD; c += 4) *reinterpret_cast<float4*>(po + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+            if (half == 0) {
+                float* pm = p.part_ml + (((size_t)split * p.max_nodes + row) * p.heads + h) * 2;
+                pm[0] = m * 0.6931471805599453f;               // back to the natural-log domain the merge kernel uses
+                pm[1] = l + sm->xl[r ^ 64];
             }
         }
     } else {
@@ -436,7 +582,8 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         return GHD_EINVAL;
     }
     CUtensorMap tm_q, tm_k, tm_v;
-    if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, QM, &tm_q) ||
+    const bool pair = n <= 64;                           // two threads per query row (queries loaded twice)
+    if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, pair ? 64 : QM, &tm_q) ||
         !tmap_planes(c, kv->k, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_k) ||
         !tmap_planes(c, kv->v, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_v)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: tensor map encoding failed");
@@ -459,16 +606,24 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
     dim3 grid(splits, H, mtiles);
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(k_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<64>()) != cudaSuccess ||
-            cudaFuncSetAttribute(k_attn_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<128>()) != cudaSuccess) {
+        const int b64 = (int)attn_smem_bytes<64>(), b128 = (int)attn_smem_bytes<128>();
+        if (cudaFuncSetAttribute(k_attn_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 attention: cannot raise dynamic shared memory");
             cudaGetLastError();
             return GHD_ECUDA;
         }
         attr_set = true;
     }
-    if (dh == 64) launch_k(c, true, k_attn_tc<64>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
-    else launch_k(c, true, k_attn_tc<128>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
+    if (dh == 64) {
+        if (pair) launch_k(c, true, k_attn_tc<64, true>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
+        else launch_k(c, true, k_attn_tc<64, false>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
+    } else {
+        if (pair) launch_k(c, true, k_attn_tc<128, true>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
+        else launch_k(c, true, k_attn_tc<128, false>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
+    }
     launch_attn_combine(c, out, splits, n);
     return GHD_OK;
 }
