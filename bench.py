@@ -174,6 +174,16 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def slowest_rank(times, dist, device):
+    """Replicas run independently; the job is as slow as its slowest rank: element-wise max over ranks."""
+    if dist is None:
+        return list(times)
+    import torch
+    t = torch.tensor(list(times), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 # ---------------------------------------------------------------- GPU arm
 def run_gpu(args):
     import torch
@@ -288,10 +298,7 @@ def run_gpu(args):
     kern_bytes = 2 * f * d * 2 + n * d * 2 + n * 2 * f * 4
     peak, peak_kind = measured_peak()
 
-    if dist is not None:
-        t = torch.tensor([ms_per_step, e2e_ms, kern_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms, kern_ms = t.tolist()
+    ms_per_step, e2e_ms, kern_ms = slowest_rank([ms_per_step, e2e_ms, kern_ms], dist, "cuda")
 
     if rank == 0:
         step_bytes = algorithmic_bytes(shape, n, kv_len)
