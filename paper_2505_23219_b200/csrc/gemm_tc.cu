@@ -468,6 +468,19 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     const long long total = (long long)p.n_tiles * p.kiters;
     int ctas = c->opt_gemm_ctas > 0 ? c->opt_gemm_ctas : c->sm_count;
     if (ctas > c->sm_count) ctas = c->sm_count;
+    if (c->opt_gemm_ctas <= 0 && epi.mode != EPI_DEFER && p.n_tiles < c->sm_count) {
+        // Fewer tiles than SMs: every CTA range is shorter than a tile.  With n_tiles * q / (q - 1) CTAs each
+        // range is (q-1)/q of a tile and always touches a tile boundary, so no tile is shared by three CTAs
+        // and no CTA's only unit sits strictly inside a tile (those finish together and take the slow
+        // split-tile path).  Take the largest such count that fits the SMs.
+        int best = 0;
+        for (int q = 2; q <= 64; ++q)
+            if ((p.n_tiles * q) % (q - 1) == 0) {
+                const int g = p.n_tiles * q / (q - 1);
+                if (g <= c->sm_count && g > best) best = g;
+            }
+        if (best >= c->sm_count * 3 / 4) ctas = best;
+    }
     if (ctas > total) ctas = (int)total;
     const size_t smem = smem_bytes_for(p.nb, p.ks, p.stages);
     static bool attr_set = false;
