@@ -433,7 +433,7 @@ bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
         const int kch = (k / TILE_K + ks - 1) / ks;
         const long long total = (long long)n_tiles * kch;
         if (ctas > total) ctas = (int)total;
-        if (m % 4 || m > 16384 || total / ctas + 1 > kch) return false;
+        if (m % 4 || m > 16384 || total / ctas + 1 > kch || total / ctas < 1) return false;
     }
     return true;
 }
@@ -502,6 +502,14 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
         c->pending.total = total;
         c->pending.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
         c->pending.m = m;
+        for (int t = 0; t < p.n_tiles && t < 128; ++t) {
+            const long long t_first = (long long)t * p.kiters;
+            const int c_first = (int)(((t_first + 1) * ctas + total - 1) / total) - 1;
+            const int c_last = (int)(((t_first + p.kiters) * ctas + total - 1) / total) - 1;
+            c->pending.first_cta[t] = (unsigned short)c_first;
+            c->pending.n_contrib[t] = (unsigned char)(c_last - c_first + 1);
+            c->pending.first_slot[t] = (total * c_first / ctas >= t_first) ? 0 : 1;
+        }
     }
     launch_k(c, true, k_gemm_tc, ctas, THREADS, smem, tm_w, tm_x, p);
     return GHD_OK;

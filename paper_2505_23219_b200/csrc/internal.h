@@ -53,6 +53,10 @@ struct PendingPartials {
     int active, kiters, ctas, m;
     long long total;
     size_t slot_elems;
+    // per 128-row tile, worked out on the host (integer divisions are expensive on the device):
+    // first contributing CTA, number of contributors, and the slot of the first one (later ones use slot 0)
+    unsigned short first_cta[128];
+    unsigned char n_contrib[128], first_slot[128];
 };
 
 }  // namespace ghd

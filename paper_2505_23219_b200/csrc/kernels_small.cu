@@ -240,19 +240,16 @@ __global__ void __launch_bounds__(1024) k_fold_pending(float* __restrict__ xres,
         v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (idx < nv) {
             const int f = 4 * idx, tile = f >> 7, row = f & 127;
-            const long long t_first = (long long)tile * pp.kiters;
-            const int c_first = (int)(((t_first + 1) * pp.ctas + pp.total - 1) / pp.total) - 1;
-            const int c_last = (int)(((t_first + pp.kiters) * pp.ctas + pp.total - 1) / pp.total) - 1;
+            const int c_first = pp.first_cta[tile], cnt = pp.n_contrib[tile], slot0 = pp.first_slot[tile];
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int cb = c_first; cb <= c_last; cb += 8) {          // up to eight loads in flight, summed in CTA order
+            for (int cb = 0; cb < cnt; cb += 8) {          // up to eight loads in flight, summed in CTA order
                 float4 t[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
-                    const int c = cb + q;
                     t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (c <= c_last) {
-                        const int slot = (pp.total * c / pp.ctas >= t_first) ? 0 : 1;
-                        t[q] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)c * 2 + slot) * pp.slot_elems +
+                    if (cb + q < cnt) {
+                        const int slot = (cb + q == 0) ? slot0 : 0;
+                        t[q] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(c_first + cb + q) * 2 + slot) * pp.slot_elems +
                                                                       (size_t)node * 128 + row));
                     }
                 }
