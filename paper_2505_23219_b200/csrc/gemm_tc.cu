@@ -39,6 +39,7 @@ constexpr int UMMA_K = 16;           // k per tcgen05.mma of kind::f16
 constexpr int MAX_STAGES = 10;
 constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
 constexpr int THREADS = 192;
+constexpr int MAX_TILES = 256;
 
 struct GemmParams {
     int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
@@ -49,17 +50,15 @@ struct GemmParams {
     int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
     int* status;
     EpiArgs epi;
+    // per tile, worked out on the host (64-bit divisions are slow on the device): first contributing
+    // CTA, number of contributors, slot of the first contributor (the others use slot 0)
+    unsigned short tile_first[MAX_TILES];
+    unsigned char tile_count[MAX_TILES], tile_slot[MAX_TILES];
 };
 
 using namespace tc;
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// First CTA whose iteration range contains flattened iteration `it` (ranges are
-// [total*c/G, total*(c+1)/G) and G <= total, so none is empty).
-__device__ __forceinline__ int cta_of_iter(long long it, long long total, int G) {
-    return (int)(((it + 1) * G + total - 1) / total) - 1;
-}
 
 struct Smem {
     uint64_t full[MAX_STAGES];
@@ -259,8 +258,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             long long units = 0;
             bool ok = true;
             long long it = it_beg;
+            int tile = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)tile * p.kiters);   // later units: next tile, k0 = 0
             while (it < it_end && ok) {
-                const int tile = (int)(it / p.kiters), k0 = (int)(it - (long long)tile * p.kiters);
                 const long long left = it_end - it;
                 const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
                 if (units >= 2) ok = mbar_wait(smem_u32(&sm->tmem_empty[buf]), buf_phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMEM);
@@ -287,6 +286,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 ++units;
                 if (++buf == 2) { buf = 0; buf_phase ^= 1; }
                 it += (k1 - k0);
+                ++tile;
+                k0 = 0;
             }
             if (!ok) {
                 // make sure no MMA is still running before TMEM goes away
@@ -304,8 +305,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         bool ok = true;
         long long it = it_beg;
         const size_t slot_elems = (size_t)buf_cols * TILE_M;   // columns padded to whole 32-wide chunks
-        while (it < it_end && ok) {
-            const int tile = (int)(it / p.kiters), k0 = (int)(it - (long long)tile * p.kiters);
+        int tile = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)tile * p.kiters);
+        for (; it < it_end && ok; ++tile, k0 = 0) {
             const long long left = it_end - it;
             const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
             const bool whole = (k0 == 0 && k1 == p.kiters) && p.epi.mode != EPI_DEFER;
@@ -329,8 +330,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 // its only unit of this tile), slot 1 when it is the head part of the CTA's last tile
                 const int slot = (it == it_beg) ? 0 : 1;
                 float* mine = p.part + ((size_t)cta * 2 + slot) * slot_elems;
-                const long long t_first = (long long)tile * p.kiters;
-                const int c_first = cta_of_iter(t_first, total, G), c_last = cta_of_iter(t_first + p.kiters - 1, total, G);
+                const int c_first = p.tile_first[tile], c_last = c_first + p.tile_count[tile] - 1;
                 bool finish = false;       // this CTA completes the tile
                 bool dumped = false;
                 if (p.epi.mode != EPI_DEFER) {
@@ -376,8 +376,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                                 for (int j = 0; j < 32; ++j) v[j] += own[j];
                                 continue;
                             }
-                            const long long cb = total * c / G;
-                            const int cslot = (cb >= t_first) ? 0 : 1;
+                            const int cslot = (c == c_first) ? p.tile_slot[tile] : 0;
                             const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems + (size_t)c0 * TILE_M + row;
                             float t[32];
 #pragma unroll
@@ -424,7 +423,7 @@ int pick_stages(int nb, int ks) {
 bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
     if (c->cfg.dtype != GHD_F16 || n < 1 || n > GHD_MAX_NODES || k % TILE_K || k < TILE_K) return false;
     const int n_tiles = (epi_mode == EPI_SWIGLU) ? (m / 2) / 64 : (m + TILE_M - 1) / TILE_M;
-    if (n_tiles < 1 || n_tiles > 4096) return false;
+    if (n_tiles < 1 || n_tiles > MAX_TILES) return false;
     if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
     if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
     if (epi_mode == EPI_DEFER) {
@@ -490,6 +489,14 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
             return GHD_ECUDA;
         }
         attr_set = true;
+    }
+    for (int t = 0; t < p.n_tiles; ++t) {
+        const long long t_first = (long long)t * p.kiters;
+        const int c_first = (int)(((t_first + 1) * ctas + total - 1) / total) - 1;
+        const int c_last = (int)(((t_first + p.kiters) * ctas + total - 1) / total) - 1;
+        p.tile_first[t] = (unsigned short)c_first;
+        p.tile_count[t] = (unsigned char)(c_last - c_first + 1);
+        p.tile_slot[t] = (total * c_first / ctas >= t_first) ? 0 : 1;
     }
     if (epi.mode == EPI_DEFER) {
         if (total / ctas + 1 > p.kiters) {                // a CTA range must touch at most two tiles
