@@ -132,26 +132,43 @@ __global__ void k_attn_combine(const float* __restrict__ part_o, const float* __
 // Same merge, one block per node and four consecutive features per thread (16-byte loads):
 // used when the row width is a multiple of 4, i.e. always for the supported head sizes.
 template <typename T>
-__global__ void k_attn_combine_rows(const float* __restrict__ part_o, const float* __restrict__ part_ml, T* __restrict__ out,
+__global__ void __launch_bounds__(1024) k_attn_combine_rows(const float* __restrict__ part_o, const float* __restrict__ part_ml, T* __restrict__ out,
                                     int splits, int heads, int dh, int max_nodes) {
     pdl_wait();
     pdl_trigger();
     const int i = blockIdx.x, d = heads * dh;
     for (int f = 4 * threadIdx.x; f < d; f += 4 * blockDim.x) {
         const int h = f / dh;
-        float ms[16], m = -INFINITY;
-        for (int s = 0; s < splits; ++s) {
-            ms[s] = part_ml[(((size_t)s * max_nodes + i) * heads + h) * 2];
-            m = fmaxf(m, ms[s]);
-        }
-        float den = 0.f;
+        // all loads of up to four splits go out together, then the weights are worked out
+        float ms[4], ls[4];
+        float4 ov[4];
+        float m = -INFINITY, den = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < splits; ++s) {
-            if (ms[s] == -INFINITY) continue;
-            const float w = expf(ms[s] - m);
-            den += part_ml[(((size_t)s * max_nodes + i) * heads + h) * 2 + 1] * w;
-            const float4 o = *reinterpret_cast<const float4*>(part_o + ((size_t)s * max_nodes + i) * d + f);
-            acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+        for (int s0 = 0; s0 < splits; s0 += 4) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int s = s0 + q;
+                ms[q] = -INFINITY; ls[q] = 0.f; ov[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (s < splits) {
+                    const float2 ml = *reinterpret_cast<const float2*>(part_ml + (((size_t)s * max_nodes + i) * heads + h) * 2);
+                    ms[q] = ml.x; ls[q] = ml.y;
+                    ov[q] = *reinterpret_cast<const float4*>(part_o + ((size_t)s * max_nodes + i) * d + f);
+                }
+            }
+            float m_new = m;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) m_new = fmaxf(m_new, ms[q]);
+            if (m_new == -INFINITY) continue;
+            const float rescale = (m == -INFINITY) ? 0.f : expf(m - m_new);
+            den *= rescale; acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (ms[q] == -INFINITY) continue;
+                const float w = expf(ms[q] - m_new);
+                den += ls[q] * w;
+                acc.x += ov[q].x * w; acc.y += ov[q].y * w; acc.z += ov[q].z * w; acc.w += ov[q].w * w;
+            }
+            m = m_new;
         }
         const float inv = 1.f / den;
         T* dst = out + (size_t)i * d + f;
