@@ -218,6 +218,9 @@ def run_gpu(args):
                        shape.dtype, shape.rms_eps, shape.rope_theta)
     ctx = ghd.ghd_create(cfg)
     ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, 2)
+    for spec in args.opt:
+        o, v = spec.split("=")
+        ghd.ghd_set_option(ctx, int(o), int(v))
     tree = ghd.Tree(ctx)
     tok_d = dev(tokens)
     amax_d = torch.empty(n, dtype=torch.int32, device="cuda")
@@ -343,6 +346,7 @@ def main():
     ap.add_argument("--kv-len", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (default 32)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--opt", action="append", default=[], metavar="ID=VALUE", help="ghd_set_option knob for sweeps (repeatable)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -56,8 +56,18 @@ typedef enum ghd_option {
                                  CUDA graph captured on first use for the same arguments    */
     GHD_OPT_GEMM_CTAS = 4,    /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
     GHD_OPT_GEMM_BURST = 5,   /* k-steps whose weight loads the tcgen05 GEMM issues together  */
-    GHD_OPT_NO_PDL = 6        /* 1 = launch every kernel fully serialised (no programmatic
+    GHD_OPT_NO_PDL = 6,       /* 1 = launch every kernel fully serialised (no programmatic
                                  dependent launch overlap between consecutive kernels)        */
+    GHD_OPT_CHAIN = 7,        /* 1 = the projections of a layer and the element-wise steps between
+                                 them run as ONE persistent kernel whose CTAs hand over through
+                                 grid-wide phase counters (GHD_F16, tcgen05 paths, d_model % 128
+                                 == 0); 0 = one kernel per projection (default: it measures
+                                 faster on a B200)                                              */
+    GHD_OPT_CHAIN_COOP = 8,   /* 0 auto / 2 = launch that kernel as a cooperative grid, 1 = plain */
+    GHD_OPT_GEMM_EVEN = 9     /* 0 = every tcgen05 projection uses the stream-K tile kernel (default);
+                                 1 = wide projections of <= 64 nodes deal their output rows evenly
+                                 to the SMs and never split the reduction; 2 + mask = the same for
+                                 the epilogues in mask only (1 plain, 2 SwiGLU, 4 RoPE/KV append)  */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary
@@ -133,6 +143,30 @@ size_t ghd_workspace_bytes(const ghd_ctx *ctx);
  * the one-time clearing of the parts that must start at zero. */
 ghd_status ghd_set_workspace(ghd_ctx *ctx, void *dev_ptr, size_t bytes);
 ghd_status ghd_set_option(ghd_ctx *ctx, int32_t option, int32_t value);
+
+/* Diagnostics (no counterpart in the paper): how many launches so far went to each kernel family,
+ * so that a test can tell which path really ran. */
+typedef enum ghd_path {
+    GHD_PATH_GEMM_TILE = 0,   /* tcgen05 projection, stream-K over 128-row tiles      */
+    GHD_PATH_GEMM_EVEN = 1,   /* tcgen05 projection, rows dealt evenly, no k-split    */
+    GHD_PATH_GEMM_SIMT = 2,   /* CUDA-core projection                                 */
+    GHD_PATH_ATTN_TC = 3,     /* tcgen05 tree attention                               */
+    GHD_PATH_ATTN_SIMT = 4,   /* CUDA-core tree attention                             */
+    GHD_PATH_CHAIN = 5        /* persistent projection-chain kernel                   */
+} ghd_path;
+int64_t ghd_path_count(const ghd_ctx *ctx, int32_t path);
+
+/* Diagnostics (no counterpart in the paper): phase time stamps of the persistent projection-chain
+ * kernel.  `dev_ptr` (dev, caller-owned, 8-byte aligned, at least ghd_trace_bytes) receives, for
+ * every launch of that kernel, int64 nanosecond stamps laid out [phase 0..8][CTA][8]:
+ * 0 epilogue warps reach the phase, 1 their dependency wait ends (element-wise phase) / the last
+ * accumulator of the phase is complete (projection), 2 their work ends, 3 the activation
+ * producer's dependency wait ends, 4 / 5 first / last weight tile requested, 6 last activation
+ * tile requested, 7 first accumulator complete; row [8][CTA][0] holds the CTA's start.  Each launch
+ * overwrites the last.
+ * NULL switches tracing off (the default).  GHD_ENOSPACE when the buffer is too small. */
+size_t ghd_trace_bytes(const ghd_ctx *ctx);
+ghd_status ghd_set_trace(ghd_ctx *ctx, void *dev_ptr, size_t bytes);
 
 /* Sec. II-C / III-C-1 (verification tree): parent_host[n], parent[0] = -1,
  * 0 <= parent[i] < i.  Fills tree->mask/parent/depth/pos/rope (see ghd_tree).

@@ -573,7 +573,7 @@ bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t) {
     return c->cfg.dtype == GHD_F16 && (c->cfg.d_head == 64 || c->cfg.d_head == 128) && t->n >= 1;
 }
 
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, int* splits_out) {
     const ghd_model_cfg& m = c->cfg;
     const int n = t->n, H = m.n_heads, dh = m.d_head, d = m.d_model;
     const int kt = t->kv_len + n;
@@ -624,7 +624,8 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         if (pair) launch_k(c, true, k_attn_tc<128, true>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
         else launch_k(c, true, k_attn_tc<128, false>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
     }
-    launch_attn_combine(c, out, splits, n);
+    if (splits_out) *splits_out = splits;
+    else launch_attn_combine(c, out, splits, n);
     return GHD_OK;
 }
 

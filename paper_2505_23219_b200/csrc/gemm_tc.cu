@@ -26,135 +26,13 @@
 #include <cstdio>
 #include <cstring>
 
-#include "internal.h"
-#include "tc_common.cuh"
+#include "gemm_tc_dev.cuh"
 
 namespace ghd {
 
+using namespace gemmdev;
+
 namespace {
-
-constexpr int TILE_M = 128;          // output features per tile (MMA M)
-constexpr int TILE_K = 64;           // halfs per k-step = one 128-byte swizzle row
-constexpr int UMMA_K = 16;           // k per tcgen05.mma of kind::f16
-constexpr int MAX_STAGES = 10;
-constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
-constexpr int THREADS = 192;
-constexpr int MAX_TILES = 256;
-
-struct GemmParams {
-    int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
-    int n_tiles, kiters, stages;     // kiters = k-chunks per tile; a chunk = ks column slabs of 64 = one pipeline stage
-    int ks, kslabs;                  // slabs per stage, slabs per weight row (k / 64)
-    int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
-    float* part;                     // [ctas][2][nb][128] float partial tiles
-    int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
-    int* status;
-    EpiArgs epi;
-    // per tile, worked out on the host (64-bit divisions are slow on the device): first contributing
-    // CTA, number of contributors, slot of the first contributor (the others use slot 0)
-    unsigned short tile_first[MAX_TILES];
-    unsigned char tile_count[MAX_TILES], tile_slot[MAX_TILES];
-};
-
-using namespace tc;
-
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-struct Smem {
-    uint64_t full[MAX_STAGES];
-    uint64_t empty[MAX_STAGES];
-    uint64_t tmem_full[2];
-    uint64_t tmem_empty[2];
-    uint64_t drain;
-    uint32_t tmem_base;
-    int abort_flag;
-    int last_flag;
-    float stage_x[EPI_CHUNK][TILE_M + 1];   // epilogue exchange buffer (rotary pairs, gate/up pairs)
-};
-
-// ---------------------------------------------------------------- fused epilogue
-// Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature
-// for nodes c0 .. c0+31.
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, int tile, int row, int c0, float (&v)[32]) {
-    const EpiArgs& e = p.epi;
-    if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
-        const int f = tile * TILE_M + row;
-        if (f < p.m) {
-            float* dst = e.out_f32 + (size_t)c0 * p.m + f;
-            if (e.mode == EPI_RESID) {
-                // all loads first, then all stores: a load placed after a store through another
-                // pointer would have to wait for it, turning 32 round trips into a chain
-                float old[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) old[j] = (c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.m) : 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] += old[j];
-            }
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (c0 + j < p.n) dst[(size_t)j * p.m] = v[j];
-        }
-        return;
-    }
-    if (e.mode == EPI_SWIGLU) {
-        // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows.
-        // After the exchange every thread finishes 16 nodes of one feature: thread `row` takes feature
-        // row & 63 and nodes 16 * (row >> 6) ...  Inputs are gathered first, stores come last (a store
-        // between two loads would serialise them: the compiler cannot prove the pointers distinct).
-#pragma unroll
-        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
-        epi_bar();
-        const int f = row & 63, jb = (row >> 6) * 16;
-        float g[16], up[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) { g[j] = sm->stage_x[jb + j][f]; up[j] = sm->stage_x[jb + j][f + 64]; }
-        __half res[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j)      // SiLU(g) * up = g * up / (1 + 2^(-g log2 e))
-            res[j] = __float2half_rn(__fdividef(g[j] * up[j], 1.f + exp2f(-1.4426950408889634f * g[j])));
-        __half* u = (__half*)e.out_t + (size_t)(c0 + jb) * p.swiglu_f + tile * 64 + f;
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-            if (c0 + jb + j < p.n) u[(size_t)j * p.swiglu_f] = res[j];
-        epi_bar();
-        return;
-    }
-    // EPI_ROPE_KV: output features [0,d) = q, [d,2d) = k, [2d,3d) = v; tiles never straddle sections
-    const int d = e.d_model, dh = e.d_head, half = dh >> 1;
-    const int f = tile * TILE_M + row;
-    const int section = f / d, el = f - section * d;
-    const int head = el / dh, idx = el - head * dh;
-    if (section < 2) {
-        const int prow = (idx < half) ? row + half : row - half;
-        const int t = (idx < half) ? idx : idx - half;
-        const float sign = (idx < half) ? -1.f : 1.f;
-        // the table loads go out first so that their latency overlaps the exchange through shared memory
-        float2 cs[32];
-        const float2* tab = reinterpret_cast<const float2*>(e.rope + (size_t)c0 * dh + 2 * t);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) cs[j] = (c0 + j < p.n) ? __ldg(tab + (size_t)j * half) : make_float2(1.f, 0.f);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
-        epi_bar();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
-        __half* dst;
-        size_t pitch;
-        if (section == 0) { dst = (__half*)e.out_t + (size_t)c0 * d + el; pitch = (size_t)d; }
-        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx; pitch = (size_t)dh; }
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (c0 + j < p.n) dst[(size_t)j * pitch] = __float2half_rn(v[j]);
-        epi_bar();
-    } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int node = c0 + j;
-            if (node < p.n)
-                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(v[j]);
-        }
-    }
-}
 
 // ---------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(THREADS, 1)
@@ -437,12 +315,13 @@ bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
     return true;
 }
 
-ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi) {
+ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi, GemmPlan* plan) {
     if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: operands must be 16-byte aligned");
         return GHD_EINVAL;
     }
-    GemmParams p{};
+    GemmParams& p = plan->p;
+    p = GemmParams{};
     p.n = n;
     p.nb = ((n + 15) / 16) * 16;
     p.k = k;
@@ -458,9 +337,8 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     p.counters = c->counters;
     p.status = c->status;
     p.epi = epi;
-    CUtensorMap tm_w, tm_x;
-    if (!tmap_slabs(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 2 : 1, p.swiglu_f ? 64 : TILE_M, (uint32_t)p.ks, &tm_w) ||
-        !tmap_slabs(c, x, (uint64_t)n, (uint64_t)k, 1, (uint32_t)p.nb, (uint32_t)p.ks, &tm_x)) {
+    if (!tmap_slabs(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 2 : 1, p.swiglu_f ? 64 : TILE_M, (uint32_t)p.ks, &plan->tm_w) ||
+        !tmap_slabs(c, x, (uint64_t)n, (uint64_t)k, 1, (uint32_t)p.nb, (uint32_t)p.ks, &plan->tm_x)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: tensor map encoding failed");
         return GHD_ECUDA;
     }
@@ -481,15 +359,8 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
         if (best >= c->sm_count * 3 / 4) ctas = best;
     }
     if (ctas > total) ctas = (int)total;
-    const size_t smem = smem_bytes_for(p.nb, p.ks, p.stages);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
-            snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
-            return GHD_ECUDA;
-        }
-        attr_set = true;
-    }
+    p.ctas = ctas;
+    plan->smem = smem_bytes_for(p.nb, p.ks, p.stages);
     for (int t = 0; t < p.n_tiles; ++t) {
         const long long t_first = (long long)t * p.kiters;
         const int c_first = (int)(((t_first + 1) * ctas + total - 1) / total) - 1;
@@ -498,27 +369,42 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
         p.tile_count[t] = (unsigned char)(c_last - c_first + 1);
         p.tile_slot[t] = (total * c_first / ctas >= t_first) ? 0 : 1;
     }
+    plan->pending.active = 0;
     if (epi.mode == EPI_DEFER) {
         if (total / ctas + 1 > p.kiters) {                // a CTA range must touch at most two tiles
             snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: deferred reduction needs n_tiles <= CTAs");
             return GHD_EUNSUPPORTED;
         }
-        c->pending.active = 1;
-        c->pending.kiters = p.kiters;
-        c->pending.ctas = ctas;
-        c->pending.total = total;
-        c->pending.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
-        c->pending.m = m;
+        PendingPartials& pp = plan->pending;
+        pp.active = 1;
+        pp.kiters = p.kiters;
+        pp.ctas = ctas;
+        pp.total = total;
+        pp.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
+        pp.m = m;
         for (int t = 0; t < p.n_tiles && t < 128; ++t) {
-            const long long t_first = (long long)t * p.kiters;
-            const int c_first = (int)(((t_first + 1) * ctas + total - 1) / total) - 1;
-            const int c_last = (int)(((t_first + p.kiters) * ctas + total - 1) / total) - 1;
-            c->pending.first_cta[t] = (unsigned short)c_first;
-            c->pending.n_contrib[t] = (unsigned char)(c_last - c_first + 1);
-            c->pending.first_slot[t] = (total * c_first / ctas >= t_first) ? 0 : 1;
+            pp.first_cta[t] = p.tile_first[t];
+            pp.n_contrib[t] = p.tile_count[t];
+            pp.first_slot[t] = p.tile_slot[t];
         }
     }
-    launch_k(c, true, k_gemm_tc, ctas, THREADS, smem, tm_w, tm_x, p);
+    return GHD_OK;
+}
+
+ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi) {
+    GemmPlan plan;
+    const ghd_status s = plan_gemm_tc(c, x, w, n, k, m, epi, &plan);
+    if (s != GHD_OK) return s;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+            snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
+            return GHD_ECUDA;
+        }
+        attr_set = true;
+    }
+    if (plan.pending.active) c->pending = plan.pending;
+    launch_k(c, true, k_gemm_tc, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
     return GHD_OK;
 }
 

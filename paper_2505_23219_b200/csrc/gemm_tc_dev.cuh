@@ -1,0 +1,153 @@
+// Device-side pieces shared by the tcgen05 projection kernels: tile constants, the parameter
+// block of one projection, the shared-memory control block, and the fused epilogues.
+#pragma once
+
+#include "internal.h"
+#include "tc_common.cuh"
+
+namespace ghd {
+namespace gemmdev {
+
+constexpr int TILE_M = 128;          // output features per tile (MMA M)
+constexpr int TILE_K = 64;           // halfs per k-step = one 128-byte swizzle row
+constexpr int UMMA_K = 16;           // k per tcgen05.mma of kind::f16
+constexpr int MAX_STAGES = 10;
+constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
+constexpr int THREADS = 192;
+constexpr int MAX_TILES = 256;
+
+struct GemmParams {
+    int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
+    int n_tiles, kiters, stages;     // kiters = k-chunks per tile; a chunk = ks column slabs of 64 = one pipeline stage
+    int ks, kslabs;                  // slabs per stage, slabs per weight row (k / 64)
+    int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
+    int ctas;                        // CTAs that share the flattened (tile, k-chunk) space
+    float* part;                     // [ctas][2][nb][128] float partial tiles
+    int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
+    int* status;
+    EpiArgs epi;
+    // per tile, worked out on the host (64-bit divisions are slow on the device): first contributing
+    // CTA, number of contributors, slot of the first contributor (the others use slot 0)
+    unsigned short tile_first[MAX_TILES];
+    unsigned char tile_count[MAX_TILES], tile_slot[MAX_TILES];
+};
+
+using namespace tc;
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct Smem {
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int last_flag;
+    float stage_x[EPI_CHUNK][TILE_M + 1];   // epilogue exchange buffer (rotary pairs, gate/up pairs)
+};
+
+// ---------------------------------------------------------------- fused epilogue
+// Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature
+// for nodes c0 .. c0+31.  `cscale` (shared memory, or null) holds one factor per node that
+// is applied to the sums first: the 1/rms of an RMSNorm whose gain is already in the operand.
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, int tile, int row, int c0, float (&v)[32],
+                                               const float* cscale = nullptr) {
+    const EpiArgs& e = p.epi;
+    if (cscale) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] *= cscale[c0 + j];
+    }
+    if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
+        const int f = tile * TILE_M + row;
+        if (f < p.m) {
+            float* dst = e.out_f32 + (size_t)c0 * p.m + f;
+            if (e.mode == EPI_RESID) {
+                // all loads first, then all stores: a load placed after a store through another
+                // pointer would have to wait for it, turning 32 round trips into a chain
+                float old[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) old[j] = (c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.m) : 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] += old[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (c0 + j < p.n) dst[(size_t)j * p.m] = v[j];
+        }
+        return;
+    }
+    if (e.mode == EPI_SWIGLU) {
+        // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows.
+        // After the exchange every thread finishes 16 nodes of one feature: thread `row` takes feature
+        // row & 63 and nodes 16 * (row >> 6) ...  Inputs are gathered first, stores come last (a store
+        // between two loads would serialise them: the compiler cannot prove the pointers distinct).
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
+        epi_bar();
+        const int f = row & 63, jb = (row >> 6) * 16;
+        float g[16], up[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { g[j] = sm->stage_x[jb + j][f]; up[j] = sm->stage_x[jb + j][f + 64]; }
+        __half res[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j)      // SiLU(g) * up = g * up / (1 + 2^(-g log2 e))
+            res[j] = __float2half_rn(__fdividef(g[j] * up[j], 1.f + exp2f(-1.4426950408889634f * g[j])));
+        __half* u = (__half*)e.out_t + (size_t)(c0 + jb) * p.swiglu_f + tile * 64 + f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (c0 + jb + j < p.n) u[(size_t)j * p.swiglu_f] = res[j];
+        epi_bar();
+        return;
+    }
+    // EPI_ROPE_KV: output features [0,d) = q, [d,2d) = k, [2d,3d) = v; tiles never straddle sections
+    const int d = e.d_model, dh = e.d_head, half = dh >> 1;
+    const int f = tile * TILE_M + row;
+    const int section = f / d, el = f - section * d;
+    const int head = el / dh, idx = el - head * dh;
+    if (section < 2) {
+        const int prow = (idx < half) ? row + half : row - half;
+        const int t = (idx < half) ? idx : idx - half;
+        const float sign = (idx < half) ? -1.f : 1.f;
+        // the table loads go out first so that their latency overlaps the exchange through shared memory
+        float2 cs[32];
+        const float2* tab = reinterpret_cast<const float2*>(e.rope + (size_t)c0 * dh + 2 * t);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) cs[j] = (c0 + j < p.n) ? __ldg(tab + (size_t)j * half) : make_float2(1.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
+        epi_bar();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
+        __half* dst;
+        size_t pitch;
+        if (section == 0) { dst = (__half*)e.out_t + (size_t)c0 * d + el; pitch = (size_t)d; }
+        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx; pitch = (size_t)dh; }
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (c0 + j < p.n) dst[(size_t)j * pitch] = __float2half_rn(v[j]);
+        epi_bar();
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const int node = c0 + j;
+            if (node < p.n)
+                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(v[j]);
+        }
+    }
+}
+
+}  // namespace gemmdev
+
+// Host: everything one projection launch needs.  `pending` describes the partial tiles an
+// EPI_DEFER projection leaves behind (active = 0 for the other epilogues).
+struct GemmPlan {
+    gemmdev::GemmParams p;
+    CUtensorMap tm_w, tm_x;
+    size_t smem;
+    PendingPartials pending;
+};
+ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi, GemmPlan* plan);
+
+}  // namespace ghd

@@ -15,7 +15,7 @@
 namespace ghd {
 
 // Device status word values (first failure wins).
-enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_TIMEOUT_TMEM = 4 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_TIMEOUT_TMEM = 4, DEV_TIMEOUT_GRID = 5 };
 
 // Epilogues of the projection GEMMs.
 enum Epilogue : int {
@@ -34,6 +34,22 @@ struct EpiArgs {
     void* v_cache;
     const float* rope;    // [n][d_head] cos/sin pairs
     int kv_len, max_kv_len, d_head, d_model;
+};
+
+// One phase of a projection chain (chain_tc.cu): a projection, a fold of deferred partial tiles
+// into the residual stream with the following RMSNorm, or the merge of the attention KV splits.
+enum : int { CHAIN_GEMM = 1, CHAIN_FOLD = 2, CHAIN_COMBINE = 3 };
+constexpr int CHAIN_MAX_PHASES = 8, CHAIN_MAX_GEMMS = 4, CHAIN_MAX_FOLDS = 3;
+constexpr int CHAIN_SYNC_OFFSET = 1024;   // phase counters live in the counter block, past the tile counters
+
+struct ChainPhase {
+    int type;
+    // CHAIN_GEMM: y = x T [n][k] * w T [m][k]^T through epilogue `epi`
+    const void* x; const void* w; int k, m; EpiArgs epi;
+    // CHAIN_FOLD: xres += partial tiles of the last EPI_DEFER projection (fold_partials), then
+    // h_out = RMSNorm(xres) * gain (gain != null) and / or x_out = T(xres).  CHAIN_COMBINE: x_out = merged attention
+    const void* gain; void* h_out; void* x_out; int fold_partials;
+    int splits;   // CHAIN_COMBINE
 };
 
 struct TmapKey {
@@ -68,7 +84,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_chain, opt_chain_coop, opt_gemm_even;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -83,11 +99,14 @@ struct ghd_ctx {
     float* gemm_part; // float [ctas][2][256][128] split tile partial sums
     int* counters;    // int [tiles] arrival counters (zero between launches)
     float* logits;    // float [max_nodes][vocab]
+    float* ssq;       // float [max_nodes][64] per-tile shares of the rows' sums of squares (chain kernel)
     int* status;      // device status word
+    long long* trace; // caller's buffer for the chain kernel's phase time stamps, or null
     int max_splits;
     ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
     int64_t launches;
+    int64_t path_count[8];   // launches per kernel family (ghd_path)
     char err[256];
     std::map<ghd::TmapKey, std::vector<uint64_t>>* tmaps;   // cached tensor maps (128-byte blobs)
     std::vector<ghd::StepGraph*>* graphs;
@@ -148,10 +167,20 @@ void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n);   // merges 
 
 // attn_tc.cu : tcgen05 / TMA tree attention (GHD_F16 only)
 bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t);
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
+// splits_out == null: merged result in `out`; else the split partials stay in att_o / att_ml and
+// *splits_out tells how many there are (the caller merges them)
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, int* splits_out = nullptr);
 
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
 bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode);
+
+// gemm_even.cu : tcgen05 / TMA projection without k-split (rows dealt evenly to the SMs; n <= 64)
+bool gemm_even_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode);
+ghd_status launch_gemm_even(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
+
+// chain_tc.cu : several dependent phases in one persistent kernel (GHD_F16 only)
+bool chain_supported(const ghd_ctx* c, int n);
+ghd_status launch_chain(ghd_ctx* c, const ChainPhase* phases, int count, int n);
 
 }  // namespace ghd

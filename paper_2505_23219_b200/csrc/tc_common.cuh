@@ -146,6 +146,10 @@ bool tmap_rows_x_k(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, ui
 // shared memory as ks consecutive [halves*box_rows x 64] swizzled tiles.
 bool tmap_slabs(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t halves, uint32_t box_rows, uint32_t ks,
                 CUtensorMap* out);
+// Row-major weights [..][cols] seen as [cols/64][groups][planes][rows_per_plane][64] (strides in rows);
+// box = one slab x one group x all planes x box_rows x 64: the planes' rows land back to back.
+bool tmap_even(ghd_ctx* c, const void* ptr, uint64_t cols, uint32_t planes, uint64_t plane_stride_rows, uint64_t groups,
+               uint64_t group_stride_rows, uint64_t rows_per_plane, uint32_t box_rows, CUtensorMap* out);
 bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
                  uint32_t box_rows, CUtensorMap* out);
 
