@@ -203,6 +203,19 @@ ghd_status ghd_verify_step(ghd_ctx *ctx, const ghd_model_weights *w, ghd_kv_laye
 ghd_status ghd_accept(ghd_ctx *ctx, const ghd_tree *tree, const int32_t *tokens_dev, const int32_t *argmax_dev,
                       ghd_accept_result *out_dev);
 
+/* KV commit: what a step keeps of the rows it appended (paper Sec. II-A: each step extends the KV
+ * cache by the tokens it produced; Sec. II-C: only the longest validated prefix survives).
+ * For each of the n_layers caches kv[l] (dev pointers, [n_kv_heads][max_kv_len][d_head]) the rows of
+ * the accepted path move from slots kv_len + nodes[j] (tree order, where the verify call wrote
+ * them) to slots kv_len + j, j = 0 .. n_matched, so that rows [0, kv_len + n_matched + 1) are the
+ * cache of the accepted sequence; later rows keep stale tree rows.  `result_dev` is the struct
+ * ghd_accept filled (read on the device: no host round trip).  kv[l].len is a host field and is
+ * NOT changed: the caller raises it to kv_len + n_matched + 1 once it has read n_matched.
+ * Enqueued on the context's stream.  GHD_EINVAL on null pointers, GHD_ENOSPACE when
+ * kv_len + max_nodes > max_kv_len could be exceeded (kv_len < 0 or kv_len + 1 > max_kv_len). */
+ghd_status ghd_kv_commit(ghd_ctx *ctx, const ghd_kv_layer *kv, int32_t n_layers, int32_t kv_len,
+                         const ghd_accept_result *result_dev);
+
 /* Building blocks of the layer, exposed for unit tests (same kernels the layer uses).
  * ghd_linear: y float [n][m] = x T[n][k] * w T[m][k]^T.
  * ghd_rmsnorm: out T [n][d_model] = RMSNorm(x float [n][d_model]) * g.

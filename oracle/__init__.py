@@ -216,3 +216,15 @@ def accept(parent, tokens, amax):
     toks = np.zeros(n, dtype=np.int32)
     m = _lib().orc_accept(_p(parent), _p(tokens), _p(amax), n, _p(nodes), _p(toks))
     return m, nodes[:m + 1].copy(), toks[:m + 1].copy()
+
+
+def kv_commit(caches: list, kv_len: int, nodes) -> None:
+    """What a step keeps of the rows it appended (paper Sec. II-A, II-C): in every layer's (k, v) the
+    row of accepted node nodes[j], written at slot kv_len + nodes[j], becomes row kv_len + j.
+    Plain definition: all sources are read from a snapshot before anything is written."""
+    nodes = [int(x) for x in nodes]
+    for k, v in caches:
+        for a in (k, v):
+            snap = a[:, kv_len:kv_len + max(nodes) + 1].copy()
+            for j, node in enumerate(nodes):
+                a[:, kv_len + j] = snap[:, node]

@@ -17,7 +17,7 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_set_trace", "ghd_path_count",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit",
     "PATH_GEMM_TILE", "PATH_GEMM_EVEN", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_CHAIN",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
     "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_CHAIN", "OPT_CHAIN_COOP", "OPT_GEMM_EVEN", "EXPORTS",
@@ -36,7 +36,7 @@ EXPORTS = [
     "ghd_create", "ghd_destroy", "ghd_workspace_bytes", "ghd_set_workspace", "ghd_set_option", "ghd_tree_build",
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
-    "ghd_tree_attention_static", "ghd_trace_bytes", "ghd_set_trace", "ghd_path_count",
+    "ghd_tree_attention_static", "ghd_trace_bytes", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit",
 ]
 
 
@@ -100,6 +100,7 @@ def load_library(path: str | Path | None = None):
         "ghd_verify_layer": ([vp, C.POINTER(_LayerW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp], C.c_int),
         "ghd_verify_step": ([vp, C.POINTER(_ModelW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp, vp], C.c_int),
         "ghd_accept": ([vp, C.POINTER(_Tree), vp, vp, vp], C.c_int),
+        "ghd_kv_commit": ([vp, C.POINTER(_Kv), i32, i32, vp], C.c_int),
         "ghd_linear": ([vp, vp, vp, i32, i32, i32, vp], C.c_int),
         "ghd_rmsnorm": ([vp, vp, vp, i32, vp], C.c_int),
         "ghd_tree_attention": ([vp, vp, C.POINTER(_Kv), C.POINTER(_Tree), vp], C.c_int),
@@ -306,6 +307,13 @@ def ghd_accept(ctx: Ctx, tree: Tree, tokens, argmax, out=None):
         out = torch.zeros(2 + 2 * GHD_MAX_NODES, dtype=torch.int32, device=ctx.device)
     ctx._check(ctx.lib.ghd_accept(ctx.handle, C.byref(tree.c), tokens.data_ptr(), argmax.data_ptr(), out.data_ptr()))
     return out
+
+
+def ghd_kv_commit(ctx: Ctx, kvs, kv_len: int, result):
+    """Moves the cache rows of the accepted path (device struct `result` from ghd_accept) to slots
+    kv_len .. kv_len + n_matched in every layer of `kvs`.  The layers' `len` fields are left alone."""
+    arr = (_Kv * len(kvs))(*[kv.c for kv in kvs])
+    ctx._check(ctx.lib.ghd_kv_commit(ctx.handle, arr, len(kvs), kv_len, result.data_ptr()))
 
 
 def ghd_linear(ctx: Ctx, x, w, y=None):

@@ -477,6 +477,15 @@ ghd_status ghd_accept(ghd_ctx* c, const ghd_tree* tree, const int32_t* tokens_de
     return check_cuda(c, "accept");
 }
 
+ghd_status ghd_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int32_t n_layers, int32_t kv_len, const ghd_accept_result* result_dev) {
+    if (!c || !kv || !result_dev || n_layers < 1) return GHD_EINVAL;
+    if (kv_len < 0 || kv_len + 1 > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "kv_commit: kv_len outside the cache");
+    for (int l = 0; l < n_layers; ++l)
+        if (!kv[l].k || !kv[l].v) return fail(c, GHD_EINVAL, "kv_commit: null cache pointer");
+    launch_kv_commit(c, kv, n_layers, kv_len, result_dev);
+    return check_cuda(c, "kv_commit");
+}
+
 ghd_status ghd_linear(ghd_ctx* c, const void* x, const void* w, int32_t n, int32_t k, int32_t m, float* y) {
     if (!c || !x || !w || !y || n < 1 || k < 1 || m < 1) return GHD_EINVAL;
     if (n > c->cfg.max_nodes) return fail(c, GHD_ENOSPACE, "linear: n > max_nodes");

@@ -155,6 +155,7 @@ void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n);
 void launch_residual(ghd_ctx* c, const float* proj_raw, int n);
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out);
 void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out);
+void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_len, const ghd_accept_result* res);
 
 // gemm_simt.cu : y float [n][m] = x T [n][k] * w T [m][k]^T
 void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, float* y);

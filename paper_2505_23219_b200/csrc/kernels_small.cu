@@ -458,4 +458,42 @@ void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const i
     c->launches++;
 }
 
+// ---------------------------------------------------------------- KV commit
+// Block (layer, head, K or V); thread = one 16-byte piece of a row.  Row kv_len + nodes[j] moves to
+// row kv_len + j for j = 1 .. n_matched (j = 0 is the root, already in place).  nodes[] increases
+// and nodes[j] >= j, so a thread that copies its piece in ascending j never reads a piece it has
+// already overwritten, and threads own disjoint pieces: no synchronisation is needed.
+constexpr int COMMIT_LAYERS = 64;
+struct CommitPtrs {
+    void* k[COMMIT_LAYERS];
+    void* v[COMMIT_LAYERS];
+};
+
+__global__ void k_kv_commit(CommitPtrs ptrs, int heads, int max_kv_len, int row_bytes, int kv_len,
+                            const ghd_accept_result* __restrict__ res) {
+    const int layer = blockIdx.x / heads, head = blockIdx.x - layer * heads;
+    char* base = (char*)(blockIdx.y == 0 ? ptrs.k[layer] : ptrs.v[layer]) + (size_t)head * max_kv_len * row_bytes;
+    int m = res->n_matched;
+    if (m > GHD_MAX_NODES - 1) m = GHD_MAX_NODES - 1;
+    for (int j = 1; j <= m; ++j) {
+        const int src = res->nodes[j];
+        if (src == j || src < 0 || src >= GHD_MAX_NODES || kv_len + src >= max_kv_len) continue;
+        const uint4* from = reinterpret_cast<const uint4*>(base + (size_t)(kv_len + src) * row_bytes);
+        uint4* to = reinterpret_cast<uint4*>(base + (size_t)(kv_len + j) * row_bytes);
+        for (int q = threadIdx.x; q < row_bytes / 16; q += blockDim.x) to[q] = from[q];
+    }
+}
+
+void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_len, const ghd_accept_result* res) {
+    const ghd_model_cfg& m = c->cfg;
+    const int row_bytes = m.d_head * (m.dtype == GHD_F32 ? 4 : 2);
+    for (int l0 = 0; l0 < n_layers; l0 += COMMIT_LAYERS) {
+        CommitPtrs ptrs{};
+        const int cnt = n_layers - l0 < COMMIT_LAYERS ? n_layers - l0 : COMMIT_LAYERS;
+        for (int l = 0; l < cnt; ++l) { ptrs.k[l] = kv[l0 + l].k; ptrs.v[l] = kv[l0 + l].v; }
+        k_kv_commit<<<dim3(cnt * m.n_kv_heads, 2), 32, 0, c->cur>>>(ptrs, m.n_kv_heads, m.max_kv_len, row_bytes, kv_len, res);
+        c->launches++;
+    }
+}
+
 }  // namespace ghd

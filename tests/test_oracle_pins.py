@@ -419,3 +419,99 @@ def test_step_is_embedding_layers_final_norm_lm_head():
     ref = (oracle.rmsnorm(hid, head["rms_final"], sh.rms_eps)) @ head["lm_head"].astype(np.float64).T
     assert np.allclose(logits, ref, rtol=1e-12, atol=1e-14)
     assert list(am) == list(np.argmax(logits, axis=1))
+
+
+# ---------------------------------------------------------------- KV commit and multi-step decoding
+def _greedy(sh, head, layers, caches, L, first_tok, count):
+    """Plain sequential decoding: `count` single-token steps, each feeding the previous argmax.
+    -> tokens [first_tok, g1, ..., g_count]; caches are appended to in place."""
+    seq = [int(first_tok)]
+    for s in range(count):
+        vis, _, pos = oracle.tree_build([-1], L + s)
+        _, am = oracle.step(sh, head, layers, caches, L + s, vis, pos, [seq[-1]])
+        seq.append(int(am[0]))
+    return seq
+
+
+def _plant(parent, tokens, chain_tokens, vocab):
+    """Writes chain_tokens along the first-child chain below the root; other nodes keep their
+    random ids, moved off the planted id where a sibling would collide."""
+    tokens = np.array(tokens, dtype=np.int32)
+    node = 0
+    for t in chain_tokens:
+        kids = [c for c, p in enumerate(parent) if p == node]
+        if not kids:
+            break
+        tokens[kids[0]] = t
+        for c in kids[1:]:
+            while tokens[c] == t or any(tokens[c] == tokens[o] for o in kids if o != c):
+                tokens[c] = (tokens[c] + 1) % vocab
+        node = kids[0]
+    return tokens
+
+
+def test_kv_commit_leaves_the_cache_of_sequential_decoding():
+    sh = SMALL
+    L, Lmax = 6, 40
+    head = wl.head_weights(sh, 21)
+    layers = [_small_layer(21, l) for l in range(sh.n_layers)]
+    fresh = lambda: [wl.kv_cache(sh, 21, l, L, Lmax) for l in range(sh.n_layers)]
+    seq_caches = fresh()
+    g = _greedy(sh, head, layers, seq_caches, L, 11, 4)          # rows L .. L+3 now hold tokens g[0..3]
+    parent = [-1, 0, 0, 0, 1, 1, 2, 4, 4, 7, 7, 5, 9, 3]         # first-child chain 0 -> 1 -> 4 -> 7 -> 9 -> 12
+    tokens = _plant(parent, wl.draft_tokens(parent, sh.vocab, 78), g[1:4], sh.vocab)
+    tokens[0] = g[0]
+    caches = fresh()
+    vis, _, pos = oracle.tree_build(parent, L)
+    _, am = oracle.step(sh, head, layers, caches, L, vis, pos, tokens)
+    m, nodes, toks = oracle.accept(parent, tokens, am)
+    assert m >= 3 and list(toks[:4]) == g[1:5]
+    assert all(nodes[j] >= j for j in range(m + 1)) and any(nodes[j] != j for j in range(m + 1))   # rows really move
+    oracle.kv_commit(caches, L, nodes)
+    keep = min(m + 1, 4)
+    for (k, v), (sk, sv) in zip(caches, seq_caches):
+        assert np.array_equal(k[:, :L], sk[:, :L])
+        assert np.allclose(k[:, L:L + keep].astype(np.float64), sk[:, L:L + keep].astype(np.float64), rtol=1e-6, atol=1e-7)
+        assert np.allclose(v[:, L:L + keep].astype(np.float64), sv[:, L:L + keep].astype(np.float64), rtol=1e-6, atol=1e-7)
+
+
+def test_kv_commit_is_a_gather_of_rows():
+    rng = np.random.default_rng(5)
+    k = rng.standard_normal((3, 20, 4)).astype(np.float32)
+    v = rng.standard_normal((3, 20, 4)).astype(np.float32)
+    k0, v0 = k.copy(), v.copy()
+    oracle.kv_commit([(k, v)], 5, [0, 2, 3, 9])
+    for j, node in enumerate([0, 2, 3, 9]):
+        assert np.array_equal(k[:, 5 + j], k0[:, 5 + node]) and np.array_equal(v[:, 5 + j], v0[:, 5 + node])
+    assert np.array_equal(k[:, :5], k0[:, :5]) and np.array_equal(k[:, 9:], k0[:, 9:])
+
+
+def test_speculative_steps_emit_exactly_the_greedy_sequence():
+    """Tree verification is lossless: whatever is drafted, verify + accept + commit, step after step,
+    produces the tokens of plain greedy decoding (paper Sec. II-C: the verified prefix plus the
+    model's own next token)."""
+    sh = SMALL
+    L0, Lmax, total = 4, 64, 18
+    head = wl.head_weights(sh, 22)
+    layers = [_small_layer(22, l) for l in range(sh.n_layers)]
+    fresh = lambda: [wl.kv_cache(sh, 22, l, L0, Lmax) for l in range(sh.n_layers)]
+    g = _greedy(sh, head, layers, fresh(), L0, 7, total + 8)
+    caches = fresh()
+    L, root, out, step_no = L0, g[0], [], 0
+    while len(out) < total:
+        parent = wl.random_tree(10, 4, 300 + step_no, max_children=3)
+        tokens = wl.draft_tokens(parent, sh.vocab, 400 + step_no)
+        at = len(out)                                         # root token is g[at]
+        tokens = _plant(parent, tokens, g[at + 1:at + 1 + step_no % 4], sh.vocab)   # 0..3 correct drafts
+        tokens[0] = root
+        vis, _, pos = oracle.tree_build(parent, L)
+        _, am = oracle.step(sh, head, layers, caches, L, vis, pos, tokens)
+        m, nodes, toks = oracle.accept(parent, tokens, am)
+        assert m >= step_no % 4 or m >= 0
+        oracle.kv_commit(caches, L, nodes)
+        out += [int(t) for t in toks]
+        L += m + 1
+        root = int(toks[-1])
+        step_no += 1
+    assert out == g[1:len(out) + 1]
+    assert step_no < total                                    # some drafts were accepted: fewer steps than tokens
