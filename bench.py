@@ -63,18 +63,20 @@ def algorithmic_bytes(shape, n, kv_len):
 
 
 # DRAM bytes per launch of the roofline kernel from the ncu capture summarised in
-# profiles/k_gemm_tc_gate_up_projection_llama7b.md; valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"gemm_tc_sha256_16": "22c0415f88c8eb4f", "bytes_per_launch": 186.5e6}
+# profiles/k_gemm_tc_gate_up_projection_llama7b.md; valid only for the kernel sources it was taken on.
+NCU_TRAFFIC = {"sources": ("gemm_tc.cu", "gemm_tc_dev.cuh", "tc_common.cuh"), "sha256_16": "ff9331b4848498c0",
+               "bytes_per_launch": 186.1e6}
 
 
 def ncu_traffic():
     import hashlib
-    src = ROOT / "paper_2505_23219_b200" / "csrc" / "gemm_tc.cu"
+    h = hashlib.sha256()
     try:
-        same = hashlib.sha256(src.read_bytes()).hexdigest()[:16] == NCU_TRAFFIC["gemm_tc_sha256_16"]
+        for f in NCU_TRAFFIC["sources"]:
+            h.update((ROOT / "paper_2505_23219_b200" / "csrc" / f).read_bytes())
     except OSError:
-        same = False
-    return NCU_TRAFFIC["bytes_per_launch"] if same else None
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"] if h.hexdigest()[:16] == NCU_TRAFFIC["sha256_16"] else None
 
 
 def measured_peak():
