@@ -95,7 +95,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             const int my_iters = (int)(it_end - it_beg);
             // weights never change: the first few weight stages stream in while the previous kernel is still
             // finishing; the activations of those stages follow after the dependency wait
-            const int prefill = my_iters < p.stages / 2 ? my_iters : p.stages / 2;
+            const int prefill = my_iters < p.stages ? my_iters : p.stages;
             int pre_kc[MAX_STAGES];
             for (int i = 0; i < my_iters && ok; ++i) {
                 if (issued >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
