@@ -51,6 +51,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const int G = gridDim.x, cta = blockIdx.x;
     const long long total = (long long)p.n_tiles * p.kiters;
     const long long it_beg = total * cta / G, it_end = total * (cta + 1) / G;
+    const int my_iters = (int)(it_end - it_beg);
+    const int prefill = my_iters < p.stages ? my_iters : p.stages;    // weight stages requested during set-up
 
     // accumulator buffers are EPI_CHUNK-aligned so that a 32-column read never leaves the allocation
     const uint32_t buf_cols = (uint32_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK);
@@ -68,6 +70,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         sm->abort_flag = 0;
         sm->last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // This thread is also the TMA producer.  Weights never change, so the first ring-full of weight
+        // stages is requested right here: their latency overlaps the rest of the set-up (tensor-memory
+        // allocation, CTA barrier) and the tail of the preceding kernel; the activations of those stages
+        // follow after the dependency wait.
+        uint64_t pol_first;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+        int tile = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)tile * p.kiters);
+        for (int i = 0; i < prefill; ++i) {
+            const uint32_t full = smem_u32(&sm->full[i]);
+            mbar_expect_tx(full, stage_bytes);
+            tma_load_4d(tiles_addr + i * stage_bytes, &tm_w, 0, p.swiglu_f ? tile * 64 : tile * TILE_M, 0, kc * p.ks, full, pol_first);
+            if (++kc == p.kiters) { kc = 0; ++tile; }
+        }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(tmem_cols) : "memory");
@@ -92,28 +107,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             // (tile, kc) advance incrementally: a 64-bit division per stage would cost this single thread
             // more cycles than the loads it issues
             int tile = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)tile * p.kiters);
-            const int my_iters = (int)(it_end - it_beg);
-            // weights never change: the first few weight stages stream in while the previous kernel is still
-            // finishing; the activations of those stages follow after the dependency wait
-            const int prefill = my_iters < p.stages ? my_iters : p.stages;
-            int pre_kc[MAX_STAGES];
-            for (int i = 0; i < my_iters && ok; ++i) {
-                if (issued >= p.stages) ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
+            if (prefill > 0) {
+                pdl_wait();                                    // the activations belong to the preceding kernel until now
+                for (int q = 0; q < prefill; ++q) {            // activations of the stages whose weights went out during set-up
+                    tma_load_4d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, 0, 0, 0, kc * p.ks, smem_u32(&sm->full[q]), pol_keep);
+                    if (++kc == p.kiters) { kc = 0; ++tile; }
+                }
+                issued = prefill;
+                if (prefill == p.stages) phase = 1; else stage = (uint32_t)prefill;
+            }
+            for (int i = prefill; i < my_iters && ok; ++i) {
+                ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
                 if (!ok) break;
                 const uint32_t full = smem_u32(&sm->full[stage]);
                 const uint32_t a_dst = tiles_addr + stage * stage_bytes, b_dst = a_dst + a_bytes;
                 mbar_expect_tx(full, stage_bytes);
                 tma_load_4d(a_dst, &tm_w, 0, p.swiglu_f ? tile * 64 : tile * TILE_M, 0, kc * p.ks, full, pol_stream);
-                if (i < prefill) {
-                    pre_kc[i] = kc;
-                    if (i == prefill - 1) {
-                        pdl_wait();
-                        for (int q = 0; q < prefill; ++q)
-                            tma_load_4d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, 0, 0, 0, pre_kc[q] * p.ks, smem_u32(&sm->full[q]), pol_keep);
-                    }
-                } else {
-                    tma_load_4d(b_dst, &tm_x, 0, 0, 0, kc * p.ks, full, pol_keep);
-                }
+                tma_load_4d(b_dst, &tm_x, 0, 0, 0, kc * p.ks, full, pol_keep);
                 ++issued;
                 if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                 if (++kc == p.kiters) { kc = 0; ++tile; }
