@@ -35,7 +35,7 @@ using namespace gemmdev;
 namespace {
 
 // ---------------------------------------------------------------- kernel
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS_TC, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -65,7 +65,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&sm->full[s]), 1); mbar_init(smem_u32(&sm->empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), 8); }
         mbar_init(smem_u32(&sm->drain), 1);
         sm->abort_flag = 0;
         sm->last_flag = 0;
@@ -184,10 +184,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             }
         }
     } else {
-        // ------------------------------------------------ epilogue warps (TMEM lanes 32*(warp%4) ..)
-        const int quad = warp & 3;
+        // ------------------------------------------------ epilogue warps 2..9 (TMEM lanes 32*(warp%4) ..), two groups:
+        // group g = (warp - 2) / 4 takes the 32-column chunks g, g + 2, ... of every accumulator
+        const int quad = warp & 3, grp = (warp - 2) >> 2;
         const int row = quad * 32 + lane;
-        const int et = threadIdx.x - 64;                       // 0..127 among epilogue threads
+        const int et = threadIdx.x - 64;                       // 0..255 among epilogue threads
         pdl_wait();                                            // outputs, residual and partial buffers belong to earlier kernels until now
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
@@ -199,16 +200,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
             const bool whole = (k0 == 0 && k1 == p.kiters) && p.epi.mode != EPI_DEFER;
             mbar_wait(smem_u32(&sm->tmem_full[buf]), buf_phase, abort_flag, p.status, DEV_TIMEOUT_EPI);
-            epi_bar();                                         // all 128 threads take the same decision
+            all_epi_bar();                                     // all 256 threads take the same decision
             ok = (*abort_flag == 0);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
             if (whole) {
-                for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
+                for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += 2 * EPI_CHUNK) {
                     float v[32];
                     tc_ld32(t_addr + c0, v);                   // may run past nb, never past the buffer
-                    if (c0 < p.n) epilogue_chunk(p, sm, tile, row, c0, v);
+                    if (c0 < p.n) epilogue_chunk2(p, sm, grp, tile, row, c0, v);
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -226,12 +227,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     // their range, long ago: if all of them have arrived, finish the tile straight from
                     // tensor memory without the store / fence / count round trips.
                     if (et == 0) sm->last_flag = (ld_acquire_gpu(p.counters + tile) == c_last - c_first) ? 1 : 0;
-                    epi_bar();
+                    all_epi_bar();
                     finish = sm->last_flag != 0;
-                    epi_bar();
+                    all_epi_bar();
                 }
                 if (!finish) {
-                    for (int c0 = 0; c0 < p.nb; c0 += EPI_CHUNK) {
+                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += 2 * EPI_CHUNK) {
                         float v[32];
                         tc_ld32(t_addr + c0, v);
 #pragma unroll
@@ -244,15 +245,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     if (p.epi.mode != EPI_DEFER) {
                         // count this arrival: the barrier orders every thread's stores before thread 0's
                         // release, and the release is cumulative over them
-                        epi_bar();
+                        all_epi_bar();
                         if (et == 0) sm->last_flag = (atom_add_acq_rel_gpu(p.counters + tile, 1) == c_last - c_first) ? 1 : 0;
-                        epi_bar();
+                        all_epi_bar();
                         finish = sm->last_flag != 0;
-                        epi_bar();
+                        all_epi_bar();
                     }
                 }
                 if (finish) {
-                    for (int c0 = 0; c0 < p.nb && c0 < p.n; c0 += EPI_CHUNK) {
+                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += 2 * EPI_CHUNK) {
                         float v[32], own[32];
                         if (!dumped) tc_ld32(t_addr + c0, own);
 #pragma unroll
@@ -272,7 +273,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] += t[j];
                         }
-                        epilogue_chunk(p, sm, tile, row, c0, v);
+                        epilogue_chunk2(p, sm, grp, tile, row, c0, v);
                     }
                     if (!dumped) {
                         tc_fence_before();
@@ -414,7 +415,7 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
         attr_set = true;
     }
     if (plan.pending.active) c->pending = plan.pending;
-    launch_k(c, true, k_gemm_tc, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    launch_k(c, true, k_gemm_tc, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
     return GHD_OK;
 }
 
