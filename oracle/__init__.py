@@ -228,3 +228,49 @@ def kv_commit(caches: list, kv_len: int, nodes) -> None:
             snap = a[:, kv_len:kv_len + max(nodes) + 1].copy()
             for j, node in enumerate(nodes):
                 a[:, kv_len + j] = snap[:, node]
+
+
+# ---------------------------------------------------------------- verification-tree design and width choice
+# Paper Sec. III-C-1: the accuracy of a candidate sequence is estimated as the product of the calibrated
+# accuracies of its tokens; the expected acceptance length is the sum over the candidate sequences; the tree
+# for a given width is grown by adding the node of highest estimated accuracy one by one.  Sec. III-C-2 /
+# IV-C: the width is the one that maximises decoding speed, acceptance length over measured step latency.
+def arca_tree(acc, width: int):
+    """acc[l][r]: accuracy of the rank-r candidate of drafting head l (level l + 1 of the tree).
+    -> (parent list in breadth-first order, probability that each node is accepted).
+    Plain restatement: every round scans every node of the tree and every child it could still get."""
+    chosen = {(): 1.0}
+    while len(chosen) < width:
+        best = None
+        for path, prob in chosen.items():
+            if len(path) >= len(acc):
+                continue
+            for r in range(len(acc[len(path)])):
+                child = path + (r,)
+                if child in chosen:
+                    continue
+                cand = (prob * acc[len(path)][r], -len(child), tuple(-x for x in child))
+                if best is None or cand > best[0]:
+                    best = (cand, child)
+        if best is None:
+            break
+        chosen[best[1]] = best[0][0]
+    order = sorted(chosen, key=lambda p: (len(p), p))
+    index = {p: i for i, p in enumerate(order)}
+    return [-1 if not p else index[p[:-1]] for p in order], [chosen[p] for p in order]
+
+
+def expected_acceptance(node_prob) -> float:
+    """Expected tokens per step: every accepted node yields one token and the root's is certain
+    (acceptance length 1 at width 1, paper Table I)."""
+    return float(sum(node_prob))
+
+
+def best_width(latency_us: dict, acc, widths=None):
+    """-> (width with the highest expected tokens per second, {width: (tokens per step, tokens per second)})."""
+    table = {}
+    for w in (widths or sorted(latency_us)):
+        _, prob = arca_tree(acc, w)
+        tau = expected_acceptance(prob)
+        table[w] = (tau, tau / (latency_us[w] * 1e-6))
+    return max(table, key=lambda w: (table[w][1], -w)), table
