@@ -216,6 +216,35 @@ ghd_status ghd_accept(ghd_ctx *ctx, const ghd_tree *tree, const int32_t *tokens_
 ghd_status ghd_kv_commit(ghd_ctx *ctx, const ghd_kv_layer *kv, int32_t n_layers, int32_t kv_len,
                          const ghd_accept_result *result_dev);
 
+/* Self-drafting with extra heads (paper Sec. II-C: Medusa "predicts candidates for future token slots by
+ * appending additional heads at the tail" of the model; the paper's default drafter).  The paper does not
+ * spell out a head; the reading taken is the Medusa head: y_k = h + SiLU(W1_k h), logits_k = W2_k y_k, where h is
+ * the model's last hidden state (after the final RMSNorm) at the LAST ACCEPTED node, head k drafts the token
+ * k + 1 positions after the bonus token, and its top-t_k tokens (ties: lower id first) are the candidates of
+ * tree level k + 1.
+ *   w1: dev T [n_heads][d_model][d_model], w2: dev T [n_heads][vocab][d_model]. */
+typedef struct ghd_medusa_weights {
+    int32_t n_heads;                  /* <= GHD_MAX_DRAFT_HEADS */
+    const void *w1, *w2;
+} ghd_medusa_weights;
+#define GHD_MAX_DRAFT_HEADS 8
+#define GHD_MAX_TOPK 16
+
+/* Runs the heads on the hidden state that the last ghd_verify_step of this context left for node
+ * result_dev->nodes[n_matched] (read on the device) and writes, for head k, its topk_host[k] best token ids
+ * to cand_dev[k * GHD_MAX_TOPK ..] (int32, best first; unused entries -1).  logits_dev: float
+ * [n_heads][vocab] or NULL.  Must follow ghd_verify_step on the same context and stream with nothing of this
+ * library in between except ghd_accept / ghd_kv_commit.  GHD_EINVAL: null pointer, n_heads or a top-k out of
+ * range; GHD_EUNSUPPORTED with GHD_OPT_CHAIN = 1 (that path keeps the hidden state unnormalised). */
+ghd_status ghd_medusa_draft(ghd_ctx *ctx, const ghd_medusa_weights *w, const ghd_accept_result *result_dev,
+                            const int32_t *topk_host, int32_t *cand_dev, float *logits_dev);
+
+/* Fills the token slots of the next tree from the candidates: node 0 gets the bonus token
+ * result_dev->tokens[n_matched]; node i > 0 gets cand[level[i] - 1][rank[i]] (level_dev / rank_dev: int32 [n],
+ * the node's depth and its rank among the candidates of its head, e.g. from the tree design).  tokens_dev: int32 [n]. */
+ghd_status ghd_tree_fill_tokens(ghd_ctx *ctx, const int32_t *cand_dev, const ghd_accept_result *result_dev,
+                                const int32_t *level_dev, const int32_t *rank_dev, int32_t n, int32_t *tokens_dev);
+
 /* Building blocks of the layer, exposed for unit tests (same kernels the layer uses).
  * ghd_linear: y float [n][m] = x T[n][k] * w T[m][k]^T.
  * ghd_rmsnorm: out T [n][d_model] = RMSNorm(x float [n][d_model]) * g.

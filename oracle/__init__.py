@@ -274,3 +274,26 @@ def best_width(latency_us: dict, acc, widths=None):
         tau = expected_acceptance(prob)
         table[w] = (tau, tau / (latency_us[w] * 1e-6))
     return max(table, key=lambda w: (table[w][1], -w)), table
+
+
+# ---------------------------------------------------------------- drafting heads
+def medusa_draft(h, w1, w2, topk):
+    """Self-drafting heads on one hidden state h [d] (paper Sec. II-C: extra heads at the tail of the model predict
+    the tokens of the following slots; head internals as in Medusa: y_k = h + SiLU(W1_k h), logits_k = W2_k y_k).
+    w1 [K][d][d], w2 [K][V][d] in storage type, read exactly; arithmetic in float64.
+    -> (candidates: list of K int lists, best first, ties to the lower id; logits float64 [K][V])."""
+    h = np.asarray(h, dtype=np.float64)
+    cands, logits = [], []
+    for k in range(len(topk)):
+        a = np.asarray(w1[k], dtype=np.float64) @ h
+        y = h + a / (1.0 + np.exp(-a))
+        z = np.asarray(w2[k], dtype=np.float64) @ y
+        order = sorted(range(z.size), key=lambda i: (-z[i], i))
+        cands.append(order[:topk[k]])
+        logits.append(z)
+    return cands, np.stack(logits)
+
+
+def tree_fill_tokens(cands, bonus: int, level, rank):
+    """Token slots of the next tree: the root carries the bonus token, node i the rank[i]-th candidate of head level[i] - 1."""
+    return np.array([bonus] + [cands[level[i] - 1][rank[i]] for i in range(1, len(level))], dtype=np.int32)

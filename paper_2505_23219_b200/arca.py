@@ -81,7 +81,7 @@ def choose_width(latency_us: dict, acc):
     return best[0], rows
 
 
-def _measure(widths, layers, kv_len):
+def _measure(widths, layers, kv_len, draft=False):
     import sys
     from pathlib import Path
 
@@ -110,6 +110,38 @@ def _measure(widths, layers, kv_len):
     ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, 2)
     acc = synthetic_accuracies()
     lat = {}
+    draft_us = 0.0
+    if draft:
+        # the drafter of the paper's default set-up: five heads (d x d block + vocabulary projection each, random here)
+        k = len(acc)
+        mw = ghd.MedusaWeights(torch.randn(k, shape.d_model, shape.d_model, device="cuda", dtype=torch.float16) * 0.02,
+                               torch.randn(k, shape.vocab, shape.d_model, device="cuda", dtype=torch.float16) * 0.02)
+        topk = [len(a) for a in acc]
+        parent, paths, _ = build_tree(acc, 64)
+        level = dev(np.array([len(p) for p in paths], np.int32))
+        rank = dev(np.array([p[-1] if p else 0 for p in paths], np.int32))
+        tokens = dev(wl.draft_tokens(parent, shape.vocab, 5))
+        tree = ghd.ghd_tree_build(ctx, parent, kv_len)
+        amax = torch.empty(64, dtype=torch.int32, device="cuda")
+        res = torch.zeros(2 + 2 * ghd.GHD_MAX_NODES, dtype=torch.int32, device="cuda")
+        ghd.ghd_verify_step(ctx, gw, gkv, tree, tokens, logits=False, argmax=amax)
+        ghd.ghd_accept(ctx, tree, tokens, amax, res)
+        nxt = torch.empty(64, dtype=torch.int32, device="cuda")
+
+        def draft_once():
+            ghd.ghd_tree_fill_tokens(ctx, ghd.ghd_medusa_draft(ctx, mw, res, topk), res, level, rank, nxt)
+
+        for _ in range(3):
+            draft_once()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            draft_once()
+        e1.record()
+        torch.cuda.synchronize()
+        ghd.ghd_sync_status(ctx)
+        draft_us = e0.elapsed_time(e1) / 20 * 1e3
     for w in widths:
         parent, _, _ = build_tree(acc, w)
         tokens = dev(wl.draft_tokens(parent, shape.vocab, 11 + w))
@@ -132,7 +164,7 @@ def _measure(widths, layers, kv_len):
         torch.cuda.synchronize()
         ghd.ghd_sync_status(ctx)
         lat[w] = e0.elapsed_time(e1) / 20 * 1e3
-    return lat, acc
+    return lat, acc, draft_us
 
 
 def main():
@@ -141,9 +173,13 @@ def main():
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--kv-len", type=int, default=2048)
     ap.add_argument("--widths", default="1,2,4,8,16,24,32,48,64,96,128")
+    ap.add_argument("--draft", action="store_true", help="also time the five drafting heads and charge them to every width above 1")
     a = ap.parse_args()
     widths = [int(x) for x in a.widths.split(",")]
-    lat, acc = _measure(widths, a.layers, a.kv_len)
+    lat, acc, draft_us = _measure(widths, a.layers, a.kv_len, a.draft)
+    if a.draft:
+        print(f"drafting heads + token fill: {draft_us:.1f} us per step (added to the latency of every width above 1)")
+        lat = {w: l + (draft_us if w > 1 else 0.0) for w, l in lat.items()}
     best, rows = choose_width(lat, acc)
     print("| width | step latency us | expected tokens / step | tokens / s | speed-up over width 1 |")
     print("|---|---|---|---|---|")

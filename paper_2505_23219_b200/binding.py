@@ -17,7 +17,8 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
+    "MedusaWeights", "GHD_MAX_TOPK",
     "PATH_GEMM_TILE", "PATH_GEMM_EVEN", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_CHAIN",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
     "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_CHAIN", "OPT_CHAIN_COOP", "OPT_GEMM_EVEN", "EXPORTS",
@@ -25,6 +26,7 @@ __all__ = [
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
+GHD_MAX_TOPK = 16
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
 OPT_CHAIN, OPT_CHAIN_COOP, OPT_GEMM_EVEN = 7, 8, 9
 PATH_GEMM_TILE, PATH_GEMM_EVEN, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_CHAIN = 0, 1, 2, 3, 4, 5
@@ -37,6 +39,7 @@ EXPORTS = [
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
     "ghd_tree_attention_static", "ghd_trace_bytes", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit",
+    "ghd_medusa_draft", "ghd_tree_fill_tokens",
 ]
 
 
@@ -60,6 +63,10 @@ class _LayerW(C.Structure):
 class _ModelW(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("layers", C.POINTER(_LayerW)), ("rms_final", C.c_void_p),
                 ("lm_head", C.c_void_p)]
+
+
+class _MedusaW(C.Structure):
+    _fields_ = [("n_heads", C.c_int32), ("w1", C.c_void_p), ("w2", C.c_void_p)]
 
 
 class _Kv(C.Structure):
@@ -101,6 +108,8 @@ def load_library(path: str | Path | None = None):
         "ghd_verify_step": ([vp, C.POINTER(_ModelW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp, vp], C.c_int),
         "ghd_accept": ([vp, C.POINTER(_Tree), vp, vp, vp], C.c_int),
         "ghd_kv_commit": ([vp, C.POINTER(_Kv), i32, i32, vp], C.c_int),
+        "ghd_medusa_draft": ([vp, C.POINTER(_MedusaW), vp, vp, vp, vp], C.c_int),
+        "ghd_tree_fill_tokens": ([vp, vp, vp, vp, vp, i32, vp], C.c_int),
         "ghd_linear": ([vp, vp, vp, i32, i32, i32, vp], C.c_int),
         "ghd_rmsnorm": ([vp, vp, vp, i32, vp], C.c_int),
         "ghd_tree_attention": ([vp, vp, C.POINTER(_Kv), C.POINTER(_Tree), vp], C.c_int),
@@ -150,6 +159,14 @@ class ModelWeights:
         self.embed, self.layers, self.rms_final, self.lm_head = embed, list(layers), rms_final, lm_head
         self._arr = (_LayerW * max(len(self.layers), 1))(*[l.c for l in self.layers])
         self.c = _ModelW(_ptr(embed), self._arr, _ptr(rms_final), _ptr(lm_head))
+
+
+class MedusaWeights:
+    """Drafting heads: w1 [n_heads][d_model][d_model], w2 [n_heads][vocab][d_model] (device tensors)."""
+
+    def __init__(self, w1, w2):
+        self.w1, self.w2 = w1, w2
+        self.c = _MedusaW(int(w1.shape[0]), _ptr(w1), _ptr(w2))
 
 
 class KvLayer:
@@ -314,6 +331,28 @@ def ghd_kv_commit(ctx: Ctx, kvs, kv_len: int, result):
     kv_len .. kv_len + n_matched in every layer of `kvs`.  The layers' `len` fields are left alone."""
     arr = (_Kv * len(kvs))(*[kv.c for kv in kvs])
     ctx._check(ctx.lib.ghd_kv_commit(ctx.handle, arr, len(kvs), kv_len, result.data_ptr()))
+
+
+def ghd_medusa_draft(ctx: Ctx, w: MedusaWeights, result, topk, want_logits: bool = False):
+    """Candidates of the drafting heads at the last accepted node of `result` (device struct of ghd_accept).
+    -> int32 device tensor [n_heads][GHD_MAX_TOPK] (best first, -1 past a head's top-k) (+ float logits [n_heads][vocab])."""
+    topk = np.ascontiguousarray(topk, dtype=np.int32)
+    k = w.c.n_heads
+    cand = torch.empty((k, GHD_MAX_TOPK), dtype=torch.int32, device=ctx.device)
+    logits = torch.empty((k, ctx.cfg.c.vocab), dtype=torch.float32, device=ctx.device) if want_logits else None
+    ctx._check(ctx.lib.ghd_medusa_draft(ctx.handle, C.byref(w.c), result.data_ptr(), topk.ctypes.data, cand.data_ptr(),
+                                        logits.data_ptr() if want_logits else None))
+    return (cand, logits) if want_logits else cand
+
+
+def ghd_tree_fill_tokens(ctx: Ctx, cand, result, level, rank, tokens=None):
+    """tokens[0] = bonus token of `result`; tokens[i] = cand[level[i] - 1][rank[i]] (level, rank: int32 device tensors)."""
+    n = int(level.numel())
+    if tokens is None:
+        tokens = torch.empty(n, dtype=torch.int32, device=ctx.device)
+    ctx._check(ctx.lib.ghd_tree_fill_tokens(ctx.handle, cand.data_ptr(), result.data_ptr(), level.data_ptr(), rank.data_ptr(), n,
+                                            tokens.data_ptr()))
+    return tokens
 
 
 def ghd_linear(ctx: Ctx, x, w, y=None):

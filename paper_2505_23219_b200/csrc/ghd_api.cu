@@ -35,6 +35,7 @@ size_t carve_workspace(ghd_ctx* c, char* base) {
     c->gemm_part = (float*)take((size_t)c->sm_count * 2 * 256 * 128 * 4);
     c->logits = (float*)take(N * (size_t)m.vocab * 4);
     c->ssq = (float*)take(N * 64 * 4);
+    c->mlogits = (float*)take((size_t)GHD_MAX_DRAFT_HEADS * m.vocab * 4);
     return off;
 }
 
@@ -484,6 +485,44 @@ ghd_status ghd_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int32_t n_layers, i
         if (!kv[l].k || !kv[l].v) return fail(c, GHD_EINVAL, "kv_commit: null cache pointer");
     launch_kv_commit(c, kv, n_layers, kv_len, result_dev);
     return check_cuda(c, "kv_commit");
+}
+
+ghd_status ghd_medusa_draft(ghd_ctx* c, const ghd_medusa_weights* w, const ghd_accept_result* result_dev, const int32_t* topk_host,
+                            int32_t* cand_dev, float* logits_dev) {
+    if (!c || !w || !w->w1 || !w->w2 || !result_dev || !topk_host || !cand_dev) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (w->n_heads < 1 || w->n_heads > GHD_MAX_DRAFT_HEADS) return fail(c, GHD_EINVAL, "medusa: n_heads outside [1, 8]");
+    for (int k = 0; k < w->n_heads; ++k)
+        if (topk_host[k] < 1 || topk_host[k] > GHD_MAX_TOPK || topk_host[k] > c->cfg.vocab) return fail(c, GHD_EINVAL, "medusa: top-k outside [1, 16]");
+    if (c->opt_chain == 1) return fail(c, GHD_EUNSUPPORTED, "medusa: the chained path keeps the hidden state unnormalised");
+    const ghd_model_cfg& m = c->cfg;
+    const int d = m.d_model, K = w->n_heads;
+    const size_t es = m.dtype == GHD_F32 ? 4 : 2;
+    if ((size_t)K * d > (size_t)m.max_nodes * ((3 * d > 2 * m.d_ffn) ? 3 * d : 2 * m.d_ffn) || (size_t)K * d > (size_t)m.max_nodes * m.d_ffn)
+        return fail(c, GHD_ENOSPACE, "medusa: workspace too small for the heads' activations");
+    float* logits = logits_dev ? logits_dev : c->mlogits;
+    c->pending.active = 0;
+    launch_medusa_gather(c, result_dev, c->attnbuf);
+    EpiArgs e{};
+    e.mode = EPI_RAW; e.out_f32 = c->raw;
+    ghd_status s = project(c, c->attnbuf, w->w1, 1, d, K * d, e, nullptr, nullptr);      // all heads' W1 rows in one projection
+    if (s != GHD_OK) return s;
+    launch_medusa_res(c, c->attnbuf, c->raw, K, c->ubuf);
+    for (int k = 0; k < K; ++k) {
+        e.out_f32 = logits + (size_t)k * m.vocab;
+        s = project(c, (const char*)c->ubuf + (size_t)k * d * es, (const char*)w->w2 + (size_t)k * m.vocab * d * es, 1, d, m.vocab, e, nullptr, nullptr);
+        if (s != GHD_OK) return s;
+    }
+    launch_medusa_topk(c, logits, K, m.vocab, topk_host, cand_dev);
+    return check_cuda(c, "medusa_draft");
+}
+
+ghd_status ghd_tree_fill_tokens(ghd_ctx* c, const int32_t* cand_dev, const ghd_accept_result* result_dev, const int32_t* level_dev,
+                                const int32_t* rank_dev, int32_t n, int32_t* tokens_dev) {
+    if (!c || !cand_dev || !result_dev || !level_dev || !rank_dev || !tokens_dev) return GHD_EINVAL;
+    if (n < 1 || n > c->cfg.max_nodes) return fail(c, GHD_ETREE, "tree_fill: n outside [1, max_nodes]");
+    launch_tree_fill(c, cand_dev, result_dev, level_dev, rank_dev, n, tokens_dev);
+    return check_cuda(c, "tree_fill_tokens");
 }
 
 ghd_status ghd_linear(ghd_ctx* c, const void* x, const void* w, int32_t n, int32_t k, int32_t m, float* y) {

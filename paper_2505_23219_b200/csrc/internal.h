@@ -99,6 +99,7 @@ struct ghd_ctx {
     float* gemm_part; // float [ctas][2][256][128] split tile partial sums
     int* counters;    // int [tiles] arrival counters (zero between launches)
     float* logits;    // float [max_nodes][vocab]
+    float* mlogits;   // float [8][vocab] logits of the drafting heads
     float* ssq;       // float [max_nodes][64] per-tile shares of the rows' sums of squares (chain kernel)
     int* status;      // device status word
     long long* trace; // caller's buffer for the chain kernel's phase time stamps, or null
@@ -155,6 +156,11 @@ void launch_swiglu(ghd_ctx* c, const float* gu_raw, int n);
 void launch_residual(ghd_ctx* c, const float* proj_raw, int n);
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out);
 void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out);
+// drafting heads (kernels_small.cu)
+void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel);                 // h_sel T [d] = hbuf[last accepted node]
+void launch_medusa_res(ghd_ctx* c, const void* h_sel, const float* raw, int heads, void* y);        // y T [heads][d] = h + SiLU(raw)
+void launch_medusa_topk(ghd_ctx* c, const float* logits, int heads, int vocab, const int* topk, int32_t* cand);
+void launch_tree_fill(ghd_ctx* c, const int32_t* cand, const ghd_accept_result* res, const int32_t* level, const int32_t* rank, int n, int32_t* tokens);
 void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_len, const ghd_accept_result* res);
 
 // gemm_simt.cu : y float [n][m] = x T [n][k] * w T [m][k]^T

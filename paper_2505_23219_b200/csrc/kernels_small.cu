@@ -458,6 +458,122 @@ void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const i
     c->launches++;
 }
 
+// ---------------------------------------------------------------- drafting heads
+// h_sel = hidden state (after the final norm) of the last accepted node, picked on the device.
+template <typename T>
+__global__ void k_medusa_gather(const T* __restrict__ hbuf, const ghd_accept_result* __restrict__ res, int d, int max_nodes, T* __restrict__ h_sel) {
+    int m = res->n_matched;
+    if (m < 0 || m >= GHD_MAX_NODES) m = 0;
+    int node = res->nodes[m];
+    if (node < 0 || node >= max_nodes) node = 0;
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < d; j += gridDim.x * blockDim.x) h_sel[j] = hbuf[(size_t)node * d + j];
+}
+
+// y[k][j] = h[j] + SiLU(raw[k * d + j])
+template <typename T>
+__global__ void k_medusa_res(const T* __restrict__ h, const float* __restrict__ raw, int heads, int d, T* __restrict__ y) {
+    const int total = heads * d;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const float a = raw[e];
+        y[e] = from_f32<T>(to_f32<T>(h[e % d]) + a / (1.f + expf(-a)));
+    }
+}
+
+// Block k: the topk[k] largest logits of head k, best first, ties to the lower id: one block-wide
+// argmax per rank, each excluding what the earlier ranks took (a taken id is greater in the order).
+struct TopkArg { int t[GHD_MAX_DRAFT_HEADS]; };
+
+__global__ void __launch_bounds__(1024) k_medusa_topk(const float* __restrict__ logits, int vocab, TopkArg topk, int32_t* __restrict__ cand) {
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    __shared__ float last_v;
+    __shared__ int last_i;
+    const float* row = logits + (size_t)blockIdx.x * vocab;
+    const int t = topk.t[blockIdx.x];
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    if (threadIdx.x == 0) { last_v = INFINITY; last_i = -1; }
+    __syncthreads();
+    for (int r = 0; r < GHD_MAX_TOPK; ++r) {
+        if (r >= t) {
+            if (threadIdx.x == 0) cand[blockIdx.x * GHD_MAX_TOPK + r] = -1;
+            continue;
+        }
+        const float lv = last_v;
+        const int li = last_i;
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int cidx = threadIdx.x; cidx < vocab; cidx += blockDim.x) {
+            const float v = row[cidx];
+            // still available: strictly after (lv, li) in the order "greater value, then smaller id"
+            if (v < lv || (v == lv && cidx > li)) amax_merge(best, bi, v, cidx);
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            amax_merge(best, bi, ov, oi);
+        }
+        if (l == 0) { sv[w] = best; si[w] = bi; }
+        __syncthreads();
+        if (w == 0) {
+            const int nw = blockDim.x >> 5;
+            best = l < nw ? sv[l] : -INFINITY;
+            bi = l < nw ? si[l] : 0x7fffffff;
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                amax_merge(best, bi, ov, oi);
+            }
+            if (l == 0) {
+                cand[blockIdx.x * GHD_MAX_TOPK + r] = (bi == 0x7fffffff) ? -1 : bi;
+                last_v = best;
+                last_i = bi;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void k_tree_fill(const int32_t* __restrict__ cand, const ghd_accept_result* __restrict__ res, const int32_t* __restrict__ level,
+                            const int32_t* __restrict__ rank, int n, int32_t* __restrict__ tokens) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    if (i == 0) {
+        int m = res->n_matched;
+        if (m < 0 || m >= GHD_MAX_NODES) m = 0;
+        tokens[0] = res->tokens[m];
+        return;
+    }
+    const int lv = level[i], rk = rank[i];
+    tokens[i] = (lv >= 1 && lv <= GHD_MAX_DRAFT_HEADS && rk >= 0 && rk < GHD_MAX_TOPK) ? cand[(lv - 1) * GHD_MAX_TOPK + rk] : -1;
+}
+
+void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel) {
+    const int d = c->cfg.d_model;
+    GHD_DISPATCH_T(c, (k_medusa_gather<float><<<1, 1024, 0, c->cur>>>((const float*)c->hbuf, res, d, c->cfg.max_nodes, (float*)h_sel)),
+                   (k_medusa_gather<__half><<<1, 1024, 0, c->cur>>>((const __half*)c->hbuf, res, d, c->cfg.max_nodes, (__half*)h_sel)));
+    c->launches++;
+}
+
+void launch_medusa_res(ghd_ctx* c, const void* h_sel, const float* raw, int heads, void* y) {
+    const int d = c->cfg.d_model;
+    const int g = grid_for((size_t)heads * d, 256, 8 * c->sm_count);
+    GHD_DISPATCH_T(c, (k_medusa_res<float><<<g, 256, 0, c->cur>>>((const float*)h_sel, raw, heads, d, (float*)y)),
+                   (k_medusa_res<__half><<<g, 256, 0, c->cur>>>((const __half*)h_sel, raw, heads, d, (__half*)y)));
+    c->launches++;
+}
+
+void launch_medusa_topk(ghd_ctx* c, const float* logits, int heads, int vocab, const int* topk, int32_t* cand) {
+    TopkArg a{};
+    for (int k = 0; k < heads; ++k) a.t[k] = topk[k];
+    k_medusa_topk<<<heads, 1024, 0, c->cur>>>(logits, vocab, a, cand);
+    c->launches++;
+}
+
+void launch_tree_fill(ghd_ctx* c, const int32_t* cand, const ghd_accept_result* res, const int32_t* level, const int32_t* rank, int n, int32_t* tokens) {
+    k_tree_fill<<<(n + 255) / 256, 256, 0, c->cur>>>(cand, res, level, rank, n, tokens);
+    c->launches++;
+}
+
 // ---------------------------------------------------------------- KV commit
 // Block (layer, head, K or V); thread = one 16-byte piece of a row.  Row kv_len + nodes[j] moves to
 // row kv_len + j for j = 1 .. n_matched (j = 0 is the root, already in place).  nodes[] increases

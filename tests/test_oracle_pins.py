@@ -515,3 +515,39 @@ def test_speculative_steps_emit_exactly_the_greedy_sequence():
         step_no += 1
     assert out == g[1:len(out) + 1]
     assert step_no < total                                    # some drafts were accepted: fewer steps than tokens
+
+
+# ---------------------------------------------------------------- drafting heads
+def test_medusa_head_closed_forms():
+    h = np.array([1.0, -2.0, 0.5])
+    eye = np.eye(3)
+    # W1 = I: y = h + h * sigmoid(h), written out; W2 = I: the logits are y itself
+    sig = 1.0 / (1.0 + np.exp(-h))
+    cands, logits = oracle.medusa_draft(h, [eye], [eye], [3])
+    assert np.allclose(logits[0], h + h * sig, rtol=1e-15)
+    assert np.allclose(logits[0], [1.7310585786300048, -2.2384058440442351, 0.8112296656009273], rtol=1e-14)   # 1 + s(1), -2 - 2 s(-2), .5 + .5 s(.5)
+    assert cands[0] == [0, 2, 1]
+    # W1 = 0: SiLU(0) = 0, the head is a plain projection of h (library matmul + stable sort as the check)
+    rng = np.random.default_rng(3)
+    h = rng.standard_normal(16)
+    w2 = rng.standard_normal((2, 40, 16)).astype(np.float32)
+    cands, logits = oracle.medusa_draft(h, np.zeros((2, 16, 16), np.float32), w2, [5, 2])
+    for k, t in enumerate([5, 2]):
+        z = w2[k].astype(np.float64) @ h
+        assert np.allclose(logits[k], z, rtol=1e-13)
+        assert cands[k] == list(np.argsort(-z, kind="stable")[:t])
+
+
+def test_medusa_topk_ties_go_to_the_lower_id():
+    h = np.array([1.0, 0.0])
+    w2 = np.array([[[0.5, 0], [2.0, 0], [2.0, 0], [0.5, 0], [3.0, 0]]])
+    cands, _ = oracle.medusa_draft(h, np.zeros((1, 2, 2)), w2, [5])
+    assert cands[0] == [4, 1, 2, 0, 3]
+
+
+def test_tree_fill_tokens_example():
+    cands = [[11, 12, 13], [21, 22], [31]]
+    #        root  L1 r0 L1 r1 L1 r2 L2 r0 (child of node 1) L2 r1  L3 r0
+    level = [0, 1, 1, 1, 2, 2, 3]
+    rank = [0, 0, 1, 2, 0, 1, 0]
+    assert list(oracle.tree_fill_tokens(cands, 99, level, rank)) == [99, 11, 12, 13, 21, 22, 31]
