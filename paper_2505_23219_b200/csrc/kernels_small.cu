@@ -17,26 +17,37 @@ template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return
 // ---------------------------------------------------------------- tree build
 struct ParentArg { int16_t p[GHD_MAX_NODES]; };
 
-// Thread i walks from node i to the root, setting one mask bit per ancestor.
-// The rotary table is computed in double so that the angle pos * theta^(-2t/dh)
-// carries no float rounding of the frequency.
+// Block b takes nodes 8b .. 8b+7: one thread per node walks to the root, setting one mask bit per
+// ancestor; then the block fills those nodes' rows of the rotary table.  The table is computed in
+// double so that the angle pos * theta^(-2t/dh) carries no float rounding of the frequency; that is
+// the slow part (pow and sincos in double), hence several blocks.
+constexpr int TREE_NODES_PER_BLOCK = 8;
+
 __global__ void k_tree_build(ParentArg pa, int n, int n_words, int kv_len, int d_head, double theta,
                              uint64_t* mask, int32_t* parent, int32_t* depth, int32_t* pos, float* rope) {
-    const int i = threadIdx.x;
-    if (i < n) {
-        uint64_t row[GHD_MAX_NODES / 64] = {0, 0, 0, 0};
-        int steps = 0;
-        for (int a = i; a >= 0 && steps <= n; a = pa.p[a]) { row[a >> 6] |= 1ull << (a & 63); ++steps; }
-        for (int w = 0; w < n_words; ++w) mask[i * n_words + w] = row[w];
-        parent[i] = pa.p[i];
-        depth[i] = steps - 1;
-        pos[i] = kv_len + steps - 1;
+    __shared__ int spos[TREE_NODES_PER_BLOCK];
+    const int first = blockIdx.x * TREE_NODES_PER_BLOCK;
+    if (threadIdx.x < TREE_NODES_PER_BLOCK) {
+        const int i = first + threadIdx.x;
+        int p = kv_len;
+        if (i < n) {
+            uint64_t row[GHD_MAX_NODES / 64] = {0, 0, 0, 0};
+            int steps = 0;
+            for (int a = i; a >= 0 && steps <= n; a = pa.p[a]) { row[a >> 6] |= 1ull << (a & 63); ++steps; }
+            for (int w = 0; w < n_words; ++w) mask[i * n_words + w] = row[w];
+            parent[i] = pa.p[i];
+            depth[i] = steps - 1;
+            p = kv_len + steps - 1;
+            pos[i] = p;
+        }
+        spos[threadIdx.x] = p;
     }
     __syncthreads();
     const int half = d_head / 2;
-    for (int e = threadIdx.x; e < n * half; e += blockDim.x) {
-        const int node = e / half, t = e % half;
-        const double ang = (double)pos[node] * pow(theta, -2.0 * t / d_head);
+    for (int e = threadIdx.x; e < TREE_NODES_PER_BLOCK * half; e += blockDim.x) {
+        const int local = e / half, t = e % half, node = first + local;
+        if (node >= n) break;
+        const double ang = (double)spos[local] * pow(theta, -2.0 * t / d_head);
         double s, c;
         sincos(ang, &s, &c);
         rope[node * d_head + 2 * t] = (float)c;
@@ -74,7 +85,7 @@ __global__ void k_tree_from_mask(int n, int n_words, int kv_len, int d_head, dou
 void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t) {
     ParentArg pa;
     for (int i = 0; i < GHD_MAX_NODES; ++i) pa.p[i] = (int16_t)(i < t->n ? parent_host[i] : -1);
-    k_tree_build<<<1, GHD_MAX_NODES, 0, c->cur>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
+    k_tree_build<<<(t->n + TREE_NODES_PER_BLOCK - 1) / TREE_NODES_PER_BLOCK, 256, 0, c->cur>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                      (double)c->cfg.rope_theta, t->mask, t->parent, t->depth,
                                                      t->pos, t->rope);
     c->launches++;
