@@ -279,6 +279,26 @@ def test_accept_bit_exact(ghd):
     ghd.ghd_sync_status(ctx)
 
 
+def test_device_wait_status_is_reported_once_and_the_context_stays_usable(ghd):
+    """A kernel whose bounded wait runs out leaves a code in the status word at the start of the workspace and
+    returns; here the word is set by hand (no kernel is made to wait): ghd_sync_status must report
+    GHD_ETIMEOUT once, clear the word, and the context must work afterwards."""
+    import torch
+    ctx = make_ctx(ghd, SMALL16, 64, 8)
+    x = wl.normal((4, 256), 1, 1.0, dtype="f16")
+    w = wl.normal((128, 256), 2, 0.02, dtype="f16")
+    y0 = ghd.ghd_linear(ctx, to_dev(x), to_dev(w))
+    ghd.ghd_sync_status(ctx)
+    ctx.workspace[:4].copy_(torch.tensor([2, 0, 0, 0], dtype=torch.uint8))      # int32 code 2 in the status word
+    with pytest.raises(ghd.GhdError) as err:
+        ghd.ghd_sync_status(ctx)
+    assert "GHD_ETIMEOUT" in str(err.value)
+    ghd.ghd_sync_status(ctx)                                                    # cleared
+    y1 = ghd.ghd_linear(ctx, to_dev(x), to_dev(w))
+    ghd.ghd_sync_status(ctx)
+    assert np.array_equal(y0.cpu().numpy(), y1.cpu().numpy())
+
+
 # ---------------------------------------------------------------- layer
 def _layer_case(ghd, shape, config_id, n, L, parent, vis=None, depth=None, gains=True, opts=()):
     Lmax = L + n
