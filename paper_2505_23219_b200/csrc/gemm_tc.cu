@@ -35,7 +35,11 @@ using namespace gemmdev;
 namespace {
 
 // ---------------------------------------------------------------- kernel
-__global__ void __launch_bounds__(THREADS_TC, 1)
+// TWO: eight epilogue warps in two groups (trees of more than 32 nodes: several 32-column chunks per tile);
+// otherwise four epilogue warps, which a single chunk cannot keep more of busy and which leaves each thread
+// the full register budget.
+template <bool TWO>
+__global__ void __launch_bounds__(TWO ? THREADS_TC : THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -65,7 +69,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&sm->full[s]), 1); mbar_init(smem_u32(&sm->empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), TWO ? 8 : 4); }
         mbar_init(smem_u32(&sm->drain), 1);
         sm->abort_flag = 0;
         sm->last_flag = 0;
@@ -186,8 +190,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     } else {
         // ------------------------------------------------ epilogue warps 2..9 (TMEM lanes 32*(warp%4) ..), two groups:
         // group g = (warp - 2) / 4 takes the 32-column chunks g, g + 2, ... of every accumulator
-        const int quad = warp & 3, grp = (warp - 2) >> 2;
+        const int quad = warp & 3, grp = TWO ? (warp - 2) >> 2 : 0;
+        constexpr int GROUPS = TWO ? 2 : 1;
         const int row = quad * 32 + lane;
+        auto epi_all = [] { if (TWO) all_epi_bar(); else epi_bar(); };
+        auto fused = [&](int tile_, int c0_, float (&v_)[32]) {
+            if (TWO) epilogue_chunk2(p, sm, grp, tile_, row, c0_, v_); else epilogue_chunk(p, sm, tile_, row, c0_, v_);
+        };
         const int et = threadIdx.x - 64;                       // 0..255 among epilogue threads
         pdl_wait();                                            // outputs, residual and partial buffers belong to earlier kernels until now
         uint32_t buf = 0, buf_phase = 0;
@@ -200,16 +209,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
             const bool whole = (k0 == 0 && k1 == p.kiters) && p.epi.mode != EPI_DEFER;
             mbar_wait(smem_u32(&sm->tmem_full[buf]), buf_phase, abort_flag, p.status, DEV_TIMEOUT_EPI);
-            all_epi_bar();                                     // all 256 threads take the same decision
+            epi_all();                                     // all 256 threads take the same decision
             ok = (*abort_flag == 0);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
             if (whole) {
-                for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += 2 * EPI_CHUNK) {
+                for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += GROUPS * EPI_CHUNK) {
                     float v[32];
                     tc_ld32(t_addr + c0, v);                   // may run past nb, never past the buffer
-                    if (c0 < p.n) epilogue_chunk2(p, sm, grp, tile, row, c0, v);
+                    if (c0 < p.n) fused(tile, c0, v);
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -227,12 +236,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     // their range, long ago: if all of them have arrived, finish the tile straight from
                     // tensor memory without the store / fence / count round trips.
                     if (et == 0) sm->last_flag = (ld_acquire_gpu(p.counters + tile) == c_last - c_first) ? 1 : 0;
-                    all_epi_bar();
+                    epi_all();
                     finish = sm->last_flag != 0;
-                    all_epi_bar();
+                    epi_all();
                 }
                 if (!finish) {
-                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += 2 * EPI_CHUNK) {
+                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += GROUPS * EPI_CHUNK) {
                         float v[32];
                         tc_ld32(t_addr + c0, v);
 #pragma unroll
@@ -245,15 +254,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     if (p.epi.mode != EPI_DEFER) {
                         // count this arrival: the barrier orders every thread's stores before thread 0's
                         // release, and the release is cumulative over them
-                        all_epi_bar();
+                        epi_all();
                         if (et == 0) sm->last_flag = (atom_add_acq_rel_gpu(p.counters + tile, 1) == c_last - c_first) ? 1 : 0;
-                        all_epi_bar();
+                        epi_all();
                         finish = sm->last_flag != 0;
-                        all_epi_bar();
+                        epi_all();
                     }
                 }
                 if (finish) {
-                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += 2 * EPI_CHUNK) {
+                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += GROUPS * EPI_CHUNK) {
                         float v[32], own[32];
                         if (!dumped) tc_ld32(t_addr + c0, own);
 #pragma unroll
@@ -273,7 +282,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] += t[j];
                         }
-                        epilogue_chunk2(p, sm, grp, tile, row, c0, v);
+                        fused(tile, c0, v);
                     }
                     if (!dumped) {
                         tc_fence_before();
@@ -408,14 +417,16 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     if (s != GHD_OK) return s;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+        if (cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
             return GHD_ECUDA;
         }
         attr_set = true;
     }
     if (plan.pending.active) c->pending = plan.pending;
-    launch_k(c, true, k_gemm_tc, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    if (plan.p.nb > EPI_CHUNK) launch_k(c, true, k_gemm_tc<true>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    else launch_k(c, true, k_gemm_tc<false>, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
     return GHD_OK;
 }
 
