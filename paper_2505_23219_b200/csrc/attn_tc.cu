@@ -32,6 +32,11 @@
 
 namespace ghd {
 
+// tmap.cu: [planes][rows_alloc][cols] tensor seen as [planes][cols/64][rows][64]; one box = (1 plane) x (all column slabs)
+// x box_rows x 64, landing as cols/64 consecutive [box_rows x 64] swizzled tiles (a row block of d_head columns per request).
+bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows, CUtensorMap* out);
+
 namespace {
 
 using namespace tc;
@@ -177,11 +182,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 const uint32_t full = smem_u32(&sm->kv_full[st]);
                 const uint32_t k_dst = kv_addr + st * STAGE_BYTES, v_dst = k_dst + SLABS * KV_SLAB;
                 mbar_expect_tx(full, STAGE_BYTES);
-#pragma unroll
-                for (int s = 0; s < SLABS; ++s) {
-                    tma_load_3d(k_dst + s * KV_SLAB, &tm_k, s * 64, key0, h, full, pol_kv);
-                    tma_load_3d(v_dst + s * KV_SLAB, &tm_v, s * 64, key0, h, full, pol_kv);
-                }
+                // one request per operand: all 64-column slabs of the 64 rows
+                tma_load_4d(k_dst, &tm_k, 0, key0, 0, h, full, pol_kv);
+                tma_load_4d(v_dst, &tm_v, 0, key0, 0, h, full, pol_kv);
             };
             // cache tiles wholly below kv_len are not written by the preceding kernel: request the
             // first ring-full of them before waiting for that kernel to finish
@@ -584,8 +587,8 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
     CUtensorMap tm_q, tm_k, tm_v;
     const bool pair = n <= 64;                           // two threads per query row (queries loaded twice)
     if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, pair ? 64 : QM, &tm_q) ||
-        !tmap_planes(c, kv->k, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_k) ||
-        !tmap_planes(c, kv->v, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_v)) {
+        !tmap_planes_slabs(c, kv->k, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_k) ||
+        !tmap_planes_slabs(c, kv->v, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, BN, &tm_v)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: tensor map encoding failed");
         return GHD_ECUDA;
     }

@@ -103,6 +103,26 @@ bool tmap_even(ghd_ctx* c, const void* ptr, uint64_t cols, uint32_t planes, uint
     return true;
 }
 
+bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows, CUtensorMap* out) {
+    const TmapKey key{ptr, rows, cols, planes, rows_alloc + (0x51abull << 48), box_rows, 64};
+    if (cached(c, key, out)) return true;
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || cols % 64) return false;
+    cuuint64_t dims[4] = {64, rows, cols / 64, planes};
+    cuuint64_t strides[3] = {cols * 2, 128, rows_alloc * cols * 2};
+    cuuint32_t box[4] = {64, box_rows, (cuuint32_t)(cols / 64), 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMap tm;
+    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    remember(c, key, tm);
+    *out = tm;
+    return true;
+}
+
 bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
                  uint32_t box_rows, CUtensorMap* out) {
     const TmapKey key{ptr, rows, cols, planes, rows_alloc, box_rows, 64};
