@@ -5,9 +5,9 @@
  * token nodes (node 0 = the root, parent[i] < i) sits on top of a KV cache of
  * length L.  One forward of the decoder stack is run for all N nodes at once;
  * node i attends to the whole cache plus only its own root-to-i ancestors
- * (Sec. II-C, Fig. 3: "a token needs to compute relationships only with
- * certain tokens"); the row argmax of the logits then decides which drafted
- * tokens are accepted (the longest validated prefix).
+ * (Sec. II-C, Fig. 3: attention between two drafted nodes is needed only
+ * along a root path); the row argmax of the logits then decides which
+ * drafted tokens are accepted (the longest validated prefix).
  *
  * Conventions
  *   - "dev" pointers are device memory on the context's GPU, "host" pointers
@@ -56,18 +56,8 @@ typedef enum ghd_option {
                                  CUDA graph captured on first use for the same arguments    */
     GHD_OPT_GEMM_CTAS = 4,    /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
     GHD_OPT_GEMM_BURST = 5,   /* k-steps whose weight loads the tcgen05 GEMM issues together  */
-    GHD_OPT_NO_PDL = 6,       /* 1 = launch every kernel fully serialised (no programmatic
+    GHD_OPT_NO_PDL = 6        /* 1 = launch every kernel fully serialised (no programmatic
                                  dependent launch overlap between consecutive kernels)        */
-    GHD_OPT_CHAIN = 7,        /* 1 = the projections of a layer and the element-wise steps between
-                                 them run as ONE persistent kernel whose CTAs hand over through
-                                 grid-wide phase counters (GHD_F16, tcgen05 paths, d_model % 128
-                                 == 0); 0 = one kernel per projection (default: it measures
-                                 faster on a B200)                                              */
-    GHD_OPT_CHAIN_COOP = 8,   /* 0 auto / 2 = launch that kernel as a cooperative grid, 1 = plain */
-    GHD_OPT_GEMM_EVEN = 9     /* 0 = every tcgen05 projection uses the stream-K tile kernel (default);
-                                 1 = wide projections of <= 64 nodes deal their output rows evenly
-                                 to the SMs and never split the reduction; 2 + mask = the same for
-                                 the epilogues in mask only (1 plain, 2 SwiGLU, 4 RoPE/KV append)  */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary
@@ -148,25 +138,11 @@ ghd_status ghd_set_option(ghd_ctx *ctx, int32_t option, int32_t value);
  * so that a test can tell which path really ran. */
 typedef enum ghd_path {
     GHD_PATH_GEMM_TILE = 0,   /* tcgen05 projection, stream-K over 128-row tiles      */
-    GHD_PATH_GEMM_EVEN = 1,   /* tcgen05 projection, rows dealt evenly, no k-split    */
-    GHD_PATH_GEMM_SIMT = 2,   /* CUDA-core projection                                 */
-    GHD_PATH_ATTN_TC = 3,     /* tcgen05 tree attention                               */
-    GHD_PATH_ATTN_SIMT = 4,   /* CUDA-core tree attention                             */
-    GHD_PATH_CHAIN = 5        /* persistent projection-chain kernel                   */
+    GHD_PATH_GEMM_SIMT = 1,   /* CUDA-core projection                                 */
+    GHD_PATH_ATTN_TC = 2,     /* tcgen05 tree attention                               */
+    GHD_PATH_ATTN_SIMT = 3    /* CUDA-core tree attention                             */
 } ghd_path;
 int64_t ghd_path_count(const ghd_ctx *ctx, int32_t path);
-
-/* Diagnostics (no counterpart in the paper): phase time stamps of the persistent projection-chain
- * kernel.  `dev_ptr` (dev, caller-owned, 8-byte aligned, at least ghd_trace_bytes) receives, for
- * every launch of that kernel, int64 nanosecond stamps laid out [phase 0..8][CTA][8]:
- * 0 epilogue warps reach the phase, 1 their dependency wait ends (element-wise phase) / the last
- * accumulator of the phase is complete (projection), 2 their work ends, 3 the activation
- * producer's dependency wait ends, 4 / 5 first / last weight tile requested, 6 last activation
- * tile requested, 7 first accumulator complete; row [8][CTA][0] holds the CTA's start.  Each launch
- * overwrites the last.
- * NULL switches tracing off (the default).  GHD_ENOSPACE when the buffer is too small. */
-size_t ghd_trace_bytes(const ghd_ctx *ctx);
-ghd_status ghd_set_trace(ghd_ctx *ctx, void *dev_ptr, size_t bytes);
 
 /* Sec. II-C / III-C-1 (verification tree): parent_host[n], parent[0] = -1,
  * 0 <= parent[i] < i.  Fills tree->mask/parent/depth/pos/rope (see ghd_tree).
@@ -216,8 +192,8 @@ ghd_status ghd_accept(ghd_ctx *ctx, const ghd_tree *tree, const int32_t *tokens_
 ghd_status ghd_kv_commit(ghd_ctx *ctx, const ghd_kv_layer *kv, int32_t n_layers, int32_t kv_len,
                          const ghd_accept_result *result_dev);
 
-/* Self-drafting with extra heads (paper Sec. II-C: Medusa "predicts candidates for future token slots by
- * appending additional heads at the tail" of the model; the paper's default drafter).  The paper does not
+/* Self-drafting with extra heads (paper Sec. II-C: Medusa-style heads attached after the last layer each
+ * draft the token of one later position; the paper's default drafter).  The paper does not
  * spell out a head; the reading taken is the Medusa head: y_k = h + SiLU(W1_k h), logits_k = W2_k y_k, where h is
  * the model's last hidden state (after the final RMSNorm) at the LAST ACCEPTED node, head k drafts the token
  * k + 1 positions after the bonus token, and its top-t_k tokens (ties: lower id first) are the candidates of
@@ -235,7 +211,7 @@ typedef struct ghd_medusa_weights {
  * to cand_dev[k * GHD_MAX_TOPK ..] (int32, best first; unused entries -1).  logits_dev: float
  * [n_heads][vocab] or NULL.  Must follow ghd_verify_step on the same context and stream with nothing of this
  * library in between except ghd_accept / ghd_kv_commit.  GHD_EINVAL: null pointer, n_heads or a top-k out of
- * range; GHD_EUNSUPPORTED with GHD_OPT_CHAIN = 1 (that path keeps the hidden state unnormalised). */
+ * range. */
 ghd_status ghd_medusa_draft(ghd_ctx *ctx, const ghd_medusa_weights *w, const ghd_accept_result *result_dev,
                             const int32_t *topk_host, int32_t *cand_dev, float *logits_dev);
 

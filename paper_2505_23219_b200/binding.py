@@ -17,19 +17,18 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
     "MedusaWeights", "GHD_MAX_TOPK",
-    "PATH_GEMM_TILE", "PATH_GEMM_EVEN", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_CHAIN",
+    "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_CHAIN", "OPT_CHAIN_COOP", "OPT_GEMM_EVEN", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
 GHD_MAX_TOPK = 16
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
-OPT_CHAIN, OPT_CHAIN_COOP, OPT_GEMM_EVEN = 7, 8, 9
-PATH_GEMM_TILE, PATH_GEMM_EVEN, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_CHAIN = 0, 1, 2, 3, 4, 5
+PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT = 0, 1, 2, 3
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
 
@@ -38,7 +37,7 @@ EXPORTS = [
     "ghd_create", "ghd_destroy", "ghd_workspace_bytes", "ghd_set_workspace", "ghd_set_option", "ghd_tree_build",
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
-    "ghd_tree_attention_static", "ghd_trace_bytes", "ghd_set_trace", "ghd_path_count", "ghd_kv_commit",
+    "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit",
     "ghd_medusa_draft", "ghd_tree_fill_tokens",
 ]
 
@@ -100,8 +99,6 @@ def load_library(path: str | Path | None = None):
         "ghd_set_workspace": ([vp, vp, C.c_size_t], C.c_int),
         "ghd_set_option": ([vp, i32, i32], C.c_int),
         "ghd_path_count": ([vp, i32], C.c_int64),
-        "ghd_trace_bytes": ([vp], C.c_size_t),
-        "ghd_set_trace": ([vp, vp, C.c_size_t], C.c_int),
         "ghd_tree_build": ([vp, vp, i32, i32, C.POINTER(_Tree)], C.c_int),
         "ghd_tree_from_mask": ([vp, vp, vp, vp, i32, i32, C.POINTER(_Tree)], C.c_int),
         "ghd_verify_layer": ([vp, C.POINTER(_LayerW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp], C.c_int),
@@ -260,19 +257,6 @@ def ghd_set_option(ctx: Ctx, option: int, value: int):
 def ghd_path_count(ctx: Ctx, path: int) -> int:
     """Launches so far that went to kernel family `path` (PATH_*)."""
     return int(ctx.lib.ghd_path_count(ctx.handle, path))
-
-
-def ghd_set_trace(ctx: Ctx, on: bool = True):
-    """Gives the context a buffer for the chain kernel's phase time stamps (or takes it away).
-    -> int64 tensor [9][SMs][8] that every chain launch overwrites, or None."""
-    if not on:
-        ctx._check(ctx.lib.ghd_set_trace(ctx.handle, None, 0))
-        ctx.trace = None
-        return None
-    nbytes = ctx.lib.ghd_trace_bytes(ctx.handle)
-    ctx.trace = torch.zeros(nbytes // 8, dtype=torch.int64, device="cuda")
-    ctx._check(ctx.lib.ghd_set_trace(ctx.handle, ctx.trace.data_ptr(), nbytes))
-    return ctx.trace.view(9, -1, 8)
 
 
 def ghd_tree_build(ctx: Ctx, parent, kv_len: int, tree: Tree | None = None) -> Tree:

@@ -32,11 +32,6 @@
 
 namespace ghd {
 
-// tmap.cu: [planes][rows_alloc][cols] tensor seen as [planes][cols/64][rows][64]; one box = (1 plane) x (all column slabs)
-// x box_rows x 64, landing as cols/64 consecutive [box_rows x 64] swizzled tiles (a row block of d_head columns per request).
-bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
-                       uint32_t box_rows, CUtensorMap* out);
-
 namespace {
 
 using namespace tc;

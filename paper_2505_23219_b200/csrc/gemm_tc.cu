@@ -193,10 +193,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         const int quad = warp & 3, grp = TWO ? (warp - 2) >> 2 : 0;
         constexpr int GROUPS = TWO ? 2 : 1;
         const int row = quad * 32 + lane;
-        auto epi_all = [] { if (TWO) all_epi_bar(); else epi_bar(); };
-        auto fused = [&](int tile_, int c0_, float (&v_)[32]) {
-            if (TWO) epilogue_chunk2(p, sm, grp, tile_, row, c0_, v_); else epilogue_chunk(p, sm, tile_, row, c0_, v_);
-        };
+        auto epi_all = [] { if (TWO) all_epi_bar(); else grp_bar(0); };
+        auto fused = [&](int tile_, int c0_, float (&v_)[32]) { epilogue_chunk<GROUPS>(p, sm, grp, tile_, row, c0_, v_); };
         const int et = threadIdx.x - 64;                       // 0..255 among epilogue threads
         pdl_wait();                                            // outputs, residual and partial buffers belong to earlier kernels until now
         uint32_t buf = 0, buf_phase = 0;

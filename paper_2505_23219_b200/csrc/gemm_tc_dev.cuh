@@ -35,8 +35,6 @@ struct GemmParams {
 
 using namespace tc;
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 struct Smem {
     uint64_t full[MAX_STAGES];
     uint64_t empty[MAX_STAGES];
@@ -50,16 +48,21 @@ struct Smem {
 };
 
 // ---------------------------------------------------------------- fused epilogue
-// Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature
-// for nodes c0 .. c0+31.  `cscale` (shared memory, or null) holds one factor per node that
-// is applied to the sums first: the 1/rms of an RMSNorm whose gain is already in the operand.
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, int tile, int row, int c0, float (&v)[32],
-                                               const float* cscale = nullptr) {
+// Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature for nodes
+// c0 .. c0+31.  GROUPS = 1: four epilogue warps; GROUPS = 2: eight epilogue warps in two groups of
+// four, group g taking the 32-column chunks g, g + 2, ... of a tile (so that the epilogue of a
+// 64-node tile takes the time of one chunk).  The rotary and SwiGLU epilogues exchange values
+// between threads through `stage_x`, XR = 32 / GROUPS node columns at a time, each group in its
+// own rows of the buffer and with its own named barrier.
+__device__ __forceinline__ void grp_bar(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory"); }
+__device__ __forceinline__ void all_epi_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+
+template <int GROUPS>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, int grp, int tile, int row, int c0, float (&v)[32]) {
+    constexpr int XR = 32 / GROUPS;      // node columns per exchange pass
+    constexpr int PASSES = GROUPS;
     const EpiArgs& e = p.epi;
-    if (cscale) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] *= cscale[c0 + j];
-    }
+    float (*xb)[TILE_M + 1] = sm->stage_x + grp * XR;
     if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
         const int f = tile * TILE_M + row;
         if (f < p.m) {
@@ -81,25 +84,29 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
     }
     if (e.mode == EPI_SWIGLU) {
         // rows 0..63: gate pre-activations of features tile*64 + row; rows 64..127: the matching up rows.
-        // After the exchange every thread finishes 16 nodes of one feature: thread `row` takes feature
-        // row & 63 and nodes 16 * (row >> 6) ...  Inputs are gathered first, stores come last (a store
-        // between two loads would serialise them: the compiler cannot prove the pointers distinct).
+        // Per pass thread `row` finishes XR/2 nodes of feature row & 63 (inputs gathered first, stores last:
+        // a store between two loads would serialise them, the compiler cannot prove the pointers distinct).
+        constexpr int HALF = XR / 2;
+        const int f = row & 63, jb = (row >> 6) * HALF;
+        __half res[PASSES * HALF];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
-        epi_bar();
-        const int f = row & 63, jb = (row >> 6) * 16;
-        float g[16], up[16];
+        for (int hh = 0; hh < PASSES; ++hh) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { g[j] = sm->stage_x[jb + j][f]; up[j] = sm->stage_x[jb + j][f + 64]; }
-        __half res[16];
+            for (int j = 0; j < XR; ++j) xb[j][row] = v[hh * XR + j];
+            grp_bar(grp);
 #pragma unroll
-        for (int j = 0; j < 16; ++j)      // SiLU(g) * up = g * up / (1 + 2^(-g log2 e))
-            res[j] = __float2half_rn(__fdividef(g[j] * up[j], 1.f + exp2f(-1.4426950408889634f * g[j])));
+            for (int j = 0; j < HALF; ++j) {      // SiLU(g) * up = g * up / (1 + 2^(-g log2 e))
+                const float g = xb[jb + j][f], up = xb[jb + j][f + 64];
+                res[hh * HALF + j] = __float2half_rn(__fdividef(g * up, 1.f + exp2f(-1.4426950408889634f * g)));
+            }
+            grp_bar(grp);
+        }
         __half* u = (__half*)e.out_t + (size_t)(c0 + jb) * p.swiglu_f + tile * 64 + f;
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-            if (c0 + jb + j < p.n) u[(size_t)j * p.swiglu_f] = res[j];
-        epi_bar();
+        for (int hh = 0; hh < PASSES; ++hh)
+#pragma unroll
+            for (int j = 0; j < HALF; ++j)
+                if (c0 + hh * XR + jb + j < p.n) u[(size_t)(hh * XR + j) * p.swiglu_f] = res[hh * HALF + j];
         return;
     }
     // EPI_ROPE_KV: output features [0,d) = q, [d,2d) = k, [2d,3d) = v; tiles never straddle sections
@@ -117,102 +124,16 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
 #pragma unroll
         for (int j = 0; j < 32; ++j) cs[j] = (c0 + j < p.n) ? __ldg(tab + (size_t)j * half) : make_float2(1.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sm->stage_x[j][row] = v[j];
-        epi_bar();
+        for (int hh = 0; hh < PASSES; ++hh) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fmaf(sign * sm->stage_x[j][prow], cs[j].y, v[j] * cs[j].x);
-        __half* dst;
-        size_t pitch;
-        if (section == 0) { dst = (__half*)e.out_t + (size_t)c0 * d + el; pitch = (size_t)d; }
-        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx; pitch = (size_t)dh; }
+            for (int j = 0; j < XR; ++j) xb[j][row] = v[hh * XR + j];
+            grp_bar(grp);
+            float partner[XR];
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (c0 + j < p.n) dst[(size_t)j * pitch] = __float2half_rn(v[j]);
-        epi_bar();
-    } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int node = c0 + j;
-            if (node < p.n)
-                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(v[j]);
-        }
-    }
-}
-
-// ---------------------------------------------------------------- the same epilogue for two groups of epilogue warps
-// k_gemm_tc runs eight epilogue warps: group g (four warps = 128 accumulator rows) takes the 32-column
-// chunks g, g + 2, ... of a tile, so that the epilogue of a 64-node tile takes the time of one chunk.
-// The groups share the exchange buffer (16 rows each) and therefore exchange 16 columns at a time.
-__device__ __forceinline__ void grp_bar(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory"); }
-__device__ __forceinline__ void all_epi_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
-
-__device__ __forceinline__ void epilogue_chunk2(const GemmParams& p, Smem* sm, int grp, int tile, int row, int c0, float (&v)[32]) {
-    const EpiArgs& e = p.epi;
-    float (*xb)[TILE_M + 1] = sm->stage_x + grp * 16;
-    if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
-        const int f = tile * TILE_M + row;
-        if (f < p.m) {
-            float* dst = e.out_f32 + (size_t)c0 * p.m + f;
-            if (e.mode == EPI_RESID) {
-                float old[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) old[j] = (c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.m) : 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] += old[j];
-            }
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (c0 + j < p.n) dst[(size_t)j * p.m] = v[j];
-        }
-        return;
-    }
-    if (e.mode == EPI_SWIGLU) {
-        // rows 0..63 gate, rows 64..127 up; per 16-column pass thread `row` finishes 8 nodes of feature row & 63
-        const int f = row & 63, jb = (row >> 6) * 8;
-        __half res[16];
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) xb[j][row] = v[hh * 16 + j];
+            for (int j = 0; j < XR; ++j) partner[j] = xb[j][prow];
             grp_bar(grp);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float g = xb[jb + j][f], up = xb[jb + j][f + 64];
-                res[hh * 8 + j] = __float2half_rn(__fdividef(g * up, 1.f + exp2f(-1.4426950408889634f * g)));
-            }
-            grp_bar(grp);
-        }
-        __half* u = (__half*)e.out_t + (size_t)(c0 + jb) * p.swiglu_f + tile * 64 + f;
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (c0 + hh * 16 + jb + j < p.n) u[(size_t)(hh * 16 + j) * p.swiglu_f] = res[hh * 8 + j];
-        return;
-    }
-    const int d = e.d_model, dh = e.d_head, half = dh >> 1;
-    const int f = tile * TILE_M + row;
-    const int section = f / d, el = f - section * d;
-    const int head = el / dh, idx = el - head * dh;
-    if (section < 2) {
-        const int prow = (idx < half) ? row + half : row - half;
-        const int t = (idx < half) ? idx : idx - half;
-        const float sign = (idx < half) ? -1.f : 1.f;
-        float2 cs[32];
-        const float2* tab = reinterpret_cast<const float2*>(e.rope + (size_t)c0 * dh + 2 * t);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) cs[j] = (c0 + j < p.n) ? __ldg(tab + (size_t)j * half) : make_float2(1.f, 0.f);
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) xb[j][row] = v[hh * 16 + j];
-            grp_bar(grp);
-            float partner[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) partner[j] = xb[j][prow];
-            grp_bar(grp);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[hh * 16 + j] = fmaf(sign * partner[j], cs[hh * 16 + j].y, v[hh * 16 + j] * cs[hh * 16 + j].x);
+            for (int j = 0; j < XR; ++j) v[hh * XR + j] = fmaf(sign * partner[j], cs[hh * XR + j].y, v[hh * XR + j] * cs[hh * XR + j].x);
         }
         __half* dst;
         size_t pitch;

@@ -34,7 +34,6 @@ size_t carve_workspace(ghd_ctx* c, char* base) {
     c->att_ml = (float*)take((size_t)c->max_splits * N * m.n_heads * 2 * 4);
     c->gemm_part = (float*)take((size_t)c->sm_count * 2 * 256 * 128 * 4);
     c->logits = (float*)take(N * (size_t)m.vocab * 4);
-    c->ssq = (float*)take(N * 64 * 4);
     c->mlogits = (float*)take((size_t)GHD_MAX_DRAFT_HEADS * m.vocab * 4);
     return off;
 }
@@ -65,14 +64,6 @@ static ghd_status project(ghd_ctx* c, const void* x, const void* w, int n, int k
     const bool tc_ok = c->cfg.dtype == GHD_F16 && gemm_tc_supported(c, n, k, m, epi.mode);
     if (c->opt_gemm_path == 2 && !tc_ok) return fail(c, GHD_EUNSUPPORTED, "tcgen05 GEMM does not take this shape/type");
     if (tc_ok && c->opt_gemm_path != 1) {
-        // measured on a B200 (7B shapes, 64 nodes): the even-rows kernel is slower than the tile kernel for the
-        // QKV and gate/up projections (its pipeline stages carry fewer weight bytes) and level for lm_head: opt-in
-        const int even_mask = c->opt_gemm_even >= 2 ? c->opt_gemm_even - 2 : (c->opt_gemm_even == 1 ? 7 : 0);
-        const int even_bit = epi.mode == EPI_RAW ? 1 : (epi.mode == EPI_SWIGLU ? 2 : 4);
-        if ((even_mask & even_bit) && gemm_even_supported(c, n, k, m, epi.mode)) {
-            c->path_count[GHD_PATH_GEMM_EVEN]++;
-            return launch_gemm_even(c, x, w, n, k, m, epi);
-        }
         c->path_count[GHD_PATH_GEMM_TILE]++;
         return launch_gemm_tc(c, x, w, n, k, m, epi);
     }
@@ -139,69 +130,6 @@ static ghd_status layer_body(ghd_ctx* c, const ghd_layer_weights* w, const ghd_k
     return GHD_OK;
 }
 
-// ---------------------------------------------------------------- chained path
-// The projections of a layer and the element-wise steps between them as phases of one persistent
-// kernel (chain_tc.cu); only the attention proper stays a kernel of its own.
-static bool chain_ok(ghd_ctx* c, const ghd_tree* t) {
-    const ghd_model_cfg& m = c->cfg;
-    const int n = t->n, d = m.d_model, f = m.d_ffn;
-    return c->opt_chain == 1 && m.dtype == GHD_F16 && c->opt_gemm_path != 1 && c->opt_attn_path != 1 && chain_supported(c, n) &&
-           attn_tc_supported(c, t) && gemm_tc_supported(c, n, d, 3 * d, EPI_ROPE_KV) && gemm_tc_supported(c, n, d, d, EPI_DEFER) &&
-           gemm_tc_supported(c, n, d, 2 * f, EPI_SWIGLU) && gemm_tc_supported(c, n, f, d, EPI_DEFER);
-}
-
-static ChainPhase ph_gemm(const void* x, const void* w, int k, int m, const EpiArgs& e) {
-    ChainPhase p{};
-    p.type = CHAIN_GEMM; p.x = x; p.w = w; p.k = k; p.m = m; p.epi = e;
-    return p;
-}
-
-static ChainPhase ph_fold(const void* gain, void* h_out, void* x_out, int fold_partials) {
-    ChainPhase p{};
-    p.type = CHAIN_FOLD; p.gain = gain; p.h_out = h_out; p.x_out = x_out; p.fold_partials = fold_partials;
-    return p;
-}
-
-static ChainPhase ph_qkv(ghd_ctx* c, const ghd_layer_weights* w, const ghd_kv_layer* kv, const ghd_tree* t) {
-    EpiArgs e = epi_base(c, t);
-    e.mode = EPI_ROPE_KV; e.out_t = c->qbuf; e.k_cache = kv->k; e.v_cache = kv->v;
-    return ph_gemm(c->hbuf, w->wqkv, c->cfg.d_model, 3 * c->cfg.d_model, e);
-}
-
-// First kernel of a stack: RMSNorm of the residual stream, then the QKV projection of its first layer.
-static ghd_status chain_head(ghd_ctx* c, const ghd_layer_weights* w, const ghd_kv_layer* kv, const ghd_tree* t) {
-    ChainPhase ph[2] = {ph_fold(w->rms1, c->hbuf, nullptr, 0), ph_qkv(c, w, kv, t)};
-    return launch_chain(c, ph, 2, t->n);
-}
-
-// Attention of a layer, then everything up to (and including, when `next` is given) the first
-// projection after the layer: split merge, O projection, fold + norm, gate/up + SwiGLU, down
-// projection, fold + the next norm (`next_gain`) and / or the layer output in storage type (`x_out`).
-static ghd_status chain_layer(ghd_ctx* c, const ghd_layer_weights* w, const ghd_kv_layer* kv, const ghd_tree* t,
-                              const void* next_gain, void* x_out, const ChainPhase* next) {
-    const ghd_model_cfg& m = c->cfg;
-    const int d = m.d_model, f = m.d_ffn;
-    int splits = 1;
-    c->path_count[GHD_PATH_ATTN_TC]++;
-    ghd_status s = launch_attn_tc(c, c->qbuf, kv, t, c->attnbuf, &splits);
-    if (s != GHD_OK) return s;
-    EpiArgs e = epi_base(c, t);
-    ChainPhase ph[CHAIN_MAX_PHASES];
-    int k = 0;
-    ph[k] = ChainPhase{};
-    ph[k].type = CHAIN_COMBINE; ph[k].x_out = c->attnbuf; ph[k].splits = splits; ++k;
-    e.mode = EPI_DEFER;
-    ph[k++] = ph_gemm(c->attnbuf, w->wo, d, d, e);
-    ph[k++] = ph_fold(w->rms2, c->hbuf, nullptr, 1);
-    e.mode = EPI_SWIGLU; e.out_t = c->ubuf;
-    ph[k++] = ph_gemm(c->hbuf, w->w_gate_up, d, 2 * f, e);
-    e.mode = EPI_DEFER; e.out_t = nullptr;
-    ph[k++] = ph_gemm(c->ubuf, w->w_down, f, d, e);
-    ph[k++] = ph_fold(next_gain, c->hbuf, x_out, 1);
-    if (next) ph[k++] = *next;
-    return launch_chain(c, ph, k, t->n);
-}
-
 static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer* kv, const ghd_tree* t,
                             const int32_t* tokens, float* logits, int32_t* amax) {
     const ghd_model_cfg& m = c->cfg;
@@ -209,29 +137,10 @@ static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer
     launch_embed(c, w->embed, tokens, t->n);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = logits;
-    if (m.n_layers > 0 && chain_ok(c, t)) {
-        if ((s = chain_head(c, &w->layers[0], &kv[0], t)) != GHD_OK) return s;
-        const bool head_in_chain = gemm_tc_supported(c, t->n, m.d_model, m.vocab, EPI_RAW);
-        for (int l = 0; l < m.n_layers; ++l) {
-            const bool last = l + 1 == m.n_layers;
-            if (last && !head_in_chain) {
-                // lm_head too wide for the chain: the layer ends with the plain fold, the final norm and
-                // the lm_head projection run as kernels of their own
-                if ((s = chain_layer(c, &w->layers[l], &kv[l], t, nullptr, nullptr, nullptr)) != GHD_OK) return s;
-                launch_rmsnorm(c, c->xres, w->rms_final, t->n, c->hbuf);
-                if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
-                break;
-            }
-            ChainPhase next = last ? ph_gemm(c->hbuf, w->lm_head, m.d_model, m.vocab, e) : ph_qkv(c, &w->layers[l + 1], &kv[l + 1], t);
-            s = chain_layer(c, &w->layers[l], &kv[l], t, last ? w->rms_final : w->layers[l + 1].rms1, nullptr, &next);
-            if (s != GHD_OK) return s;
-        }
-    } else {
-        for (int l = 0; l < m.n_layers; ++l)
-            if ((s = layer_body(c, &w->layers[l], &kv[l], t)) != GHD_OK) return s;
-        norm_into_h(c, w->rms_final, t->n);
-        if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
-    }
+    for (int l = 0; l < m.n_layers; ++l)
+        if ((s = layer_body(c, &w->layers[l], &kv[l], t)) != GHD_OK) return s;
+    norm_into_h(c, w->rms_final, t->n);
+    if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
     launch_argmax(c, logits, t->n, m.vocab, amax);
     return GHD_OK;
 }
@@ -265,10 +174,8 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->device = dev;
     c->sm_count = sms;
     c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = 0;
-    c->opt_chain = c->opt_chain_coop = c->opt_gemm_even = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
-    c->trace = nullptr;
     c->max_splits = 16;
     c->pending.active = 0;
     c->launches = 0;
@@ -307,17 +214,6 @@ ghd_status ghd_set_workspace(ghd_ctx* c, void* dev_ptr, size_t bytes) {
     return GHD_OK;
 }
 
-ghd_status ghd_set_trace(ghd_ctx* c, void* dev_ptr, size_t bytes) {
-    if (!c) return GHD_EINVAL;
-    if (dev_ptr && (bytes < ghd_trace_bytes(c) || ((uintptr_t)dev_ptr & 7))) return fail(c, GHD_ENOSPACE, "trace buffer too small or misaligned");
-    c->trace = (long long*)dev_ptr;
-    return GHD_OK;
-}
-
-size_t ghd_trace_bytes(const ghd_ctx* c) {
-    return c ? (size_t)(CHAIN_MAX_PHASES + 1) * c->sm_count * 8 * sizeof(long long) : 0;
-}
-
 ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
     if (!c || value < 0) return GHD_EINVAL;
     switch (option) {
@@ -328,9 +224,6 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
         case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
-        case GHD_OPT_CHAIN: if (value > 1) return GHD_EINVAL; c->opt_chain = value; break;
-        case GHD_OPT_GEMM_EVEN: if (value > 9) return GHD_EINVAL; c->opt_gemm_even = value; break;
-        case GHD_OPT_CHAIN_COOP: if (value > 2) return GHD_EINVAL; c->opt_chain_coop = value; break;
         default: return GHD_EINVAL;
     }
     return GHD_OK;
@@ -394,11 +287,6 @@ ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer
     if (kv->len != tree->kv_len) return fail(c, GHD_EINVAL, "layer: kv.len differs from tree.kv_len");
     c->pending.active = 0;
     launch_load_x(c, x_in, tree->n);
-    if (chain_ok(c, tree)) {
-        if ((s = chain_head(c, w, kv, tree)) != GHD_OK) return s;
-        if ((s = chain_layer(c, w, kv, tree, nullptr, x_out, nullptr)) != GHD_OK) return s;
-        return check_cuda(c, "verify_layer");
-    }
     if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
     if (c->pending.active) launch_fold_pending(c, tree->n, nullptr, nullptr, x_out);
     else launch_store_x(c, x_out, tree->n);
@@ -494,7 +382,6 @@ ghd_status ghd_medusa_draft(ghd_ctx* c, const ghd_medusa_weights* w, const ghd_a
     if (w->n_heads < 1 || w->n_heads > GHD_MAX_DRAFT_HEADS) return fail(c, GHD_EINVAL, "medusa: n_heads outside [1, 8]");
     for (int k = 0; k < w->n_heads; ++k)
         if (topk_host[k] < 1 || topk_host[k] > GHD_MAX_TOPK || topk_host[k] > c->cfg.vocab) return fail(c, GHD_EINVAL, "medusa: top-k outside [1, 16]");
-    if (c->opt_chain == 1) return fail(c, GHD_EUNSUPPORTED, "medusa: the chained path keeps the hidden state unnormalised");
     const ghd_model_cfg& m = c->cfg;
     const int d = m.d_model, K = w->n_heads;
     const size_t es = m.dtype == GHD_F32 ? 4 : 2;

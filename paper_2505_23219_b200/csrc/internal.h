@@ -36,22 +36,6 @@ struct EpiArgs {
     int kv_len, max_kv_len, d_head, d_model;
 };
 
-// One phase of a projection chain (chain_tc.cu): a projection, a fold of deferred partial tiles
-// into the residual stream with the following RMSNorm, or the merge of the attention KV splits.
-enum : int { CHAIN_GEMM = 1, CHAIN_FOLD = 2, CHAIN_COMBINE = 3 };
-constexpr int CHAIN_MAX_PHASES = 8, CHAIN_MAX_GEMMS = 4, CHAIN_MAX_FOLDS = 3;
-constexpr int CHAIN_SYNC_OFFSET = 1024;   // phase counters live in the counter block, past the tile counters
-
-struct ChainPhase {
-    int type;
-    // CHAIN_GEMM: y = x T [n][k] * w T [m][k]^T through epilogue `epi`
-    const void* x; const void* w; int k, m; EpiArgs epi;
-    // CHAIN_FOLD: xres += partial tiles of the last EPI_DEFER projection (fold_partials), then
-    // h_out = RMSNorm(xres) * gain (gain != null) and / or x_out = T(xres).  CHAIN_COMBINE: x_out = merged attention
-    const void* gain; void* h_out; void* x_out; int fold_partials;
-    int splits;   // CHAIN_COMBINE
-};
-
 struct TmapKey {
     const void* ptr; uint64_t rows, cols, planes, plane_stride; uint32_t box_rows, box_cols;
     bool operator<(const TmapKey& o) const {
@@ -84,7 +68,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_chain, opt_chain_coop, opt_gemm_even;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -100,9 +84,7 @@ struct ghd_ctx {
     int* counters;    // int [tiles] arrival counters (zero between launches)
     float* logits;    // float [max_nodes][vocab]
     float* mlogits;   // float [8][vocab] logits of the drafting heads
-    float* ssq;       // float [max_nodes][64] per-tile shares of the rows' sums of squares (chain kernel)
     int* status;      // device status word
-    long long* trace; // caller's buffer for the chain kernel's phase time stamps, or null
     int max_splits;
     ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
@@ -181,13 +163,5 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
 bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode);
-
-// gemm_even.cu : tcgen05 / TMA projection without k-split (rows dealt evenly to the SMs; n <= 64)
-bool gemm_even_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode);
-ghd_status launch_gemm_even(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
-
-// chain_tc.cu : several dependent phases in one persistent kernel (GHD_F16 only)
-bool chain_supported(const ghd_ctx* c, int n);
-ghd_status launch_chain(ghd_ctx* c, const ChainPhase* phases, int count, int n);
 
 }  // namespace ghd

@@ -139,18 +139,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 // Host: cached tensor maps (half elements, 128-byte swizzle, 64-element inner box, zero fill).
 // Row-major matrix [rows][cols] with a (box_rows x 64) box.
 bool tmap_rows_x_k(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out);
-// [planes][rows_alloc][cols] of which only the first `rows` rows of each plane are readable
-// (rows beyond read as zero); box = (1 plane x box_rows x 64).
 // Row-major [rows][cols] matrix (cols a multiple of 64) seen as [cols/64][halves][rows/halves][64]:
 // one box = (ks column slabs) x (halves) x (box_rows rows of each half) x 64 elements, which lands in
 // shared memory as ks consecutive [halves*box_rows x 64] swizzled tiles.
 bool tmap_slabs(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint32_t halves, uint32_t box_rows, uint32_t ks,
                 CUtensorMap* out);
-// Row-major weights [..][cols] seen as [cols/64][groups][planes][rows_per_plane][64] (strides in rows);
-// box = one slab x one group x all planes x box_rows x 64: the planes' rows land back to back.
-bool tmap_even(ghd_ctx* c, const void* ptr, uint64_t cols, uint32_t planes, uint64_t plane_stride_rows, uint64_t groups,
-               uint64_t group_stride_rows, uint64_t rows_per_plane, uint32_t box_rows, CUtensorMap* out);
-bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
-                 uint32_t box_rows, CUtensorMap* out);
+// [planes][rows_alloc][cols] tensor of which only the first `rows` rows of each plane are readable (rows
+// beyond read as zero), seen as [planes][cols/64][rows][64]; one box = (1 plane) x (all column slabs)
+// x box_rows x 64, landing as cols/64 consecutive [box_rows x 64] swizzled tiles.
+bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows, CUtensorMap* out);
 
 }  // namespace ghd

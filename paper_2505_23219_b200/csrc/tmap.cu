@@ -80,29 +80,6 @@ bool tmap_slabs(ghd_ctx* c, const void* ptr, uint64_t rows, uint64_t cols, uint3
     return true;
 }
 
-bool tmap_even(ghd_ctx* c, const void* ptr, uint64_t cols, uint32_t planes, uint64_t plane_stride_rows, uint64_t groups,
-               uint64_t group_stride_rows, uint64_t rows_per_plane, uint32_t box_rows, CUtensorMap* out) {
-    const TmapKey key{ptr, rows_per_plane, cols, planes, 0xe7e70000ull + (groups << 20) + (plane_stride_rows << 40) + group_stride_rows, box_rows, 64};
-    if (cached(c, key, out)) return true;
-    EncodeTiledFn fn = encode_fn();
-    if (!fn || cols % 64) return false;
-    const uint64_t row_bytes = cols * 2, whole = rows_per_plane * row_bytes;
-    cuuint64_t dims[5] = {64, rows_per_plane, planes, groups, cols / 64};
-    // a dimension of extent 1 is never stepped along: give it any legal stride
-    cuuint64_t strides[4] = {row_bytes, planes > 1 ? plane_stride_rows * row_bytes : whole,
-                             groups > 1 ? group_stride_rows * row_bytes : whole, 128};
-    cuuint32_t box[5] = {64, box_rows, planes, 1, 1};
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    CUtensorMap tm;
-    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    remember(c, key, tm);
-    *out = tm;
-    return true;
-}
-
 bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
                        uint32_t box_rows, CUtensorMap* out) {
     const TmapKey key{ptr, rows, cols, planes, rows_alloc + (0x51abull << 48), box_rows, 64};
@@ -115,26 +92,6 @@ bool tmap_planes_slabs(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t ro
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMap tm;
     if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    remember(c, key, tm);
-    *out = tm;
-    return true;
-}
-
-bool tmap_planes(ghd_ctx* c, const void* ptr, uint64_t planes, uint64_t rows_alloc, uint64_t rows, uint64_t cols,
-                 uint32_t box_rows, CUtensorMap* out) {
-    const TmapKey key{ptr, rows, cols, planes, rows_alloc, box_rows, 64};
-    if (cached(c, key, out)) return true;
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {cols, rows, planes};
-    cuuint64_t strides[2] = {cols * 2, rows_alloc * cols * 2};
-    cuuint32_t box[3] = {64, box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUtensorMap tm;
-    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
