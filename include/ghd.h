@@ -56,8 +56,10 @@ typedef enum ghd_option {
                                  CUDA graph captured on first use for the same arguments    */
     GHD_OPT_GEMM_CTAS = 4,    /* CTAs of the tcgen05 GEMM (0 = one per SM)                   */
     GHD_OPT_GEMM_BURST = 5,   /* k-steps whose weight loads the tcgen05 GEMM issues together  */
-    GHD_OPT_NO_PDL = 6        /* 1 = launch every kernel fully serialised (no programmatic
+    GHD_OPT_NO_PDL = 6,       /* 1 = launch every kernel fully serialised (no programmatic
                                  dependent launch overlap between consecutive kernels)        */
+    GHD_OPT_GEMM_STAGES = 7,  /* pipeline stages of the tcgen05 GEMM (0 = automatic)          */
+    GHD_OPT_GEMM_EPI = 8      /* epilogue warp groups of the tcgen05 GEMM: 0 auto, 1, 2        */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary

@@ -21,13 +21,14 @@ __all__ = [
     "MedusaWeights", "GHD_MAX_TOPK",
     "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
 GHD_MAX_TOPK = 16
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
+OPT_GEMM_STAGES, OPT_GEMM_EPI = 7, 8
 PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT = 0, 1, 2, 3
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]

@@ -571,7 +571,7 @@ bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t) {
     return c->cfg.dtype == GHD_F16 && (c->cfg.d_head == 64 || c->cfg.d_head == 128) && t->n >= 1;
 }
 
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, int* splits_out) {
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
     const ghd_model_cfg& m = c->cfg;
     const int n = t->n, H = m.n_heads, dh = m.d_head, d = m.d_model;
     const int kt = t->kv_len + n;
@@ -602,8 +602,7 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
     p.mask = t->mask; p.part_o = c->att_o; p.part_ml = c->att_ml; p.status = c->status;
     p.scale = 1.0f / sqrtf((float)dh);
     dim3 grid(splits, H, mtiles);
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (!c->attr_attn) {       // per context: the attribute belongs to the device the context was created on
         const int b64 = (int)attn_smem_bytes<64>(), b128 = (int)attn_smem_bytes<128>();
         if (cudaFuncSetAttribute(k_attn_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
@@ -613,7 +612,7 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
             cudaGetLastError();
             return GHD_ECUDA;
         }
-        attr_set = true;
+        c->attr_attn = true;
     }
     if (dh == 64) {
         if (pair) launch_k(c, true, k_attn_tc<64, true>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
@@ -622,8 +621,7 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         if (pair) launch_k(c, true, k_attn_tc<128, true>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
         else launch_k(c, true, k_attn_tc<128, false>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
     }
-    if (splits_out) *splits_out = splits;
-    else launch_attn_combine(c, out, splits, n);
+    launch_attn_combine(c, out, splits, n);
     return GHD_OK;
 }
 

@@ -351,6 +351,7 @@ ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, 
     p.kslabs = k / TILE_K;
     p.kiters = (p.kslabs + p.ks - 1) / p.ks;
     p.stages = pick_stages(p.nb, p.ks);
+    if (c->opt_gemm_stages >= 2 && c->opt_gemm_stages < p.stages) p.stages = c->opt_gemm_stages;
     p.part = c->gemm_part;
     p.counters = c->counters;
     p.status = c->status;
@@ -413,17 +414,17 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     GemmPlan plan;
     const ghd_status s = plan_gemm_tc(c, x, w, n, k, m, epi, &plan);
     if (s != GHD_OK) return s;
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (!c->attr_gemm) {       // per context: the attribute belongs to the device the context was created on
         if (cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
             cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
             return GHD_ECUDA;
         }
-        attr_set = true;
+        c->attr_gemm = true;
     }
     if (plan.pending.active) c->pending = plan.pending;
-    if (plan.p.nb > EPI_CHUNK) launch_k(c, true, k_gemm_tc<true>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    const bool two = c->opt_gemm_epi ? c->opt_gemm_epi == 2 : plan.p.nb > EPI_CHUNK;
+    if (two) launch_k(c, true, k_gemm_tc<true>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
     else launch_k(c, true, k_gemm_tc<false>, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
     return GHD_OK;
 }

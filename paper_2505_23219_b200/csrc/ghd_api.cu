@@ -173,11 +173,13 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
     c->pending.active = 0;
+    c->entry_fresh = 1;
+    c->attr_gemm = c->attr_attn = false;
     c->launches = 0;
     memset(c->path_count, 0, sizeof(c->path_count));
     c->tmaps = new std::map<TmapKey, std::vector<uint64_t>>();
@@ -223,6 +225,8 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_GRAPH: if (value > 2) return GHD_EINVAL; c->opt_graph = value; break;
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
         case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
+        case GHD_OPT_GEMM_STAGES: if (value == 1 || value > 10) return GHD_EINVAL; c->opt_gemm_stages = value; break;
+        case GHD_OPT_GEMM_EPI: if (value > 2) return GHD_EINVAL; c->opt_gemm_epi = value; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
         default: return GHD_EINVAL;
     }
@@ -286,6 +290,7 @@ ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer
     if (s != GHD_OK) return s;
     if (kv->len != tree->kv_len) return fail(c, GHD_EINVAL, "layer: kv.len differs from tree.kv_len");
     c->pending.active = 0;
+    c->entry_fresh = 1;
     launch_load_x(c, x_in, tree->n);
     if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
     if (c->pending.active) launch_fold_pending(c, tree->n, nullptr, nullptr, x_out);
@@ -309,6 +314,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     }
     float* logits = logits_dev ? logits_dev : c->logits;
     c->pending.active = 0;
+    c->entry_fresh = 1;
     if (c->opt_graph != 2) {
         if ((s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev)) != GHD_OK) return s;
         return check_cuda(c, "verify_step");
@@ -319,8 +325,8 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
-    key.push_back(((uint64_t)(uint32_t)c->opt_gemm_path << 48) | ((uint64_t)(uint32_t)c->opt_attn_splits << 32) |
-                  ((uint64_t)(uint32_t)c->opt_attn_path << 16) | ((uint32_t)c->opt_gemm_ctas & 0xfff) | ((uint32_t)c->opt_gemm_burst << 12) | ((uint32_t)c->opt_no_pdl << 15));
+    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi})
+        key.push_back((uint64_t)(uint32_t)o);       // every option that changes what is enqueued
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
         push(lw.wqkv); push(lw.wo); push(lw.w_gate_up); push(lw.w_down); push(lw.rms1); push(lw.rms2);
@@ -389,6 +395,7 @@ ghd_status ghd_medusa_draft(ghd_ctx* c, const ghd_medusa_weights* w, const ghd_a
         return fail(c, GHD_ENOSPACE, "medusa: workspace too small for the heads' activations");
     float* logits = logits_dev ? logits_dev : c->mlogits;
     c->pending.active = 0;
+    c->entry_fresh = 1;
     launch_medusa_gather(c, result_dev, c->attnbuf);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = c->raw;
@@ -419,12 +426,14 @@ ghd_status ghd_linear(ghd_ctx* c, const void* x, const void* w, int32_t n, int32
     if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = y;
+    c->entry_fresh = 1;
     ghd_status s = project(c, x, w, n, k, m, e, nullptr, nullptr);
     return s != GHD_OK ? s : check_cuda(c, "linear");
 }
 
 ghd_status ghd_rmsnorm(ghd_ctx* c, const float* x, const void* g, int32_t n, void* out) {
     if (!c || !x || !g || !out || n < 1) return GHD_EINVAL;
+    c->entry_fresh = 1;
     launch_rmsnorm(c, x, g, n, out);
     return check_cuda(c, "rmsnorm");
 }
@@ -434,12 +443,14 @@ ghd_status ghd_tree_attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv,
     if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
     ghd_status s = check_tree(c, tree);
     if (s != GHD_OK) return s;
+    c->entry_fresh = 1;
     if ((s = attention(c, q, kv, tree, out)) != GHD_OK) return s;
     return check_cuda(c, "tree_attention");
 }
 
 ghd_status ghd_argmax(ghd_ctx* c, const float* logits, int32_t n, int32_t v, int32_t* out) {
     if (!c || !logits || !out || n < 1 || v < 1) return GHD_EINVAL;
+    c->entry_fresh = 1;
     launch_argmax(c, logits, n, v, out);
     return check_cuda(c, "argmax");
 }

@@ -68,7 +68,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -88,6 +88,8 @@ struct ghd_ctx {
     int max_splits;
     ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
+    int entry_fresh;          // 1 until the first launch of a public call: that launch is fully serialised (see launch_k)
+    bool attr_gemm, attr_attn;  // dynamic shared memory limits raised on this context's device
     int64_t launches;
     int64_t path_count[8];   // launches per kernel family (ghd_path)
     char err[256];
@@ -106,20 +108,41 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 
+// cluster_x > 1: the CTAs of a grid row (gridDim.x a multiple of cluster_x) are launched as thread-block clusters.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_k(ghd_ctx* c, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+inline cudaError_t launch_kc(ghd_ctx* c, bool pdl, int cluster_x, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = c->cur;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (cluster_x > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster_x;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    // The first kernel of a public call is never launched programmatically: what ran before it on the
+    // stream belongs to the caller and may still be writing weights or cache rows that our kernels read
+    // ahead of their dependency wait.
+    if (pdl && !c->opt_no_pdl && !c->entry_fresh) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (pdl && !c->opt_no_pdl) ? 1 : 0;
+    cfg.numAttrs = na;
+    c->entry_fresh = 0;
     c->launches++;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(ghd_ctx* c, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+    return launch_kc(c, pdl, 1, kernel, grid, block, smem, std::forward<Args>(args)...);
 }
 
 size_t carve_workspace(ghd_ctx* c, char* base);   // returns bytes needed; assigns pointers when base != nullptr
@@ -156,9 +179,8 @@ void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n);   // merges 
 
 // attn_tc.cu : tcgen05 / TMA tree attention (GHD_F16 only)
 bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t);
-// splits_out == null: merged result in `out`; else the split partials stay in att_o / att_ml and
-// *splits_out tells how many there are (the caller merges them)
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, int* splits_out = nullptr);
+// the split partials go to att_o / att_ml and a second kernel merges them into `out`
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
 
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);
