@@ -12,9 +12,10 @@
 // and cut into equal contiguous ranges, one per CTA (one CTA per SM), so every SM
 // streams the same number of weight bytes whatever the tile count.  A CTA whose
 // range covers only part of a tile's k-steps writes its float partial tile to the
-// workspace and bumps the tile's arrival counter; whichever CTA arrives last sums
-// the partials in CTA order (fixed order -> bit-reproducible) and runs the
-// epilogue.  Nobody ever waits for another CTA.
+// workspace and bumps the tile's arrival counter; the tile's first contributor (for
+// which the tile comes last) keeps its share in tensor memory, waits - bounded - for
+// that counter, sums the partials in CTA order (fixed order -> bit-reproducible) and
+// runs the epilogue.  Contributors that store never wait.
 //
 // Per CTA: warp 0 = TMA producer (weights and activations into a ring of
 // 128B-swizzled shared-memory stages), warp 1 = MMA issuer (tcgen05.mma, one
@@ -230,10 +231,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 bool finish = false;       // this CTA completes the tile
                 bool dumped = false;
                 if (p.epi.mode != EPI_DEFER) {
-                    // Usually the other contributors handled their share of this tile as the first unit of
-                    // their range, long ago: if all of them have arrived, finish the tile straight from
-                    // tensor memory without the store / fence / count round trips.
-                    if (et == 0) sm->last_flag = (ld_acquire_gpu(p.counters + tile) == c_last - c_first) ? 1 : 0;
+                    // The tile is finished by its FIRST contributor: for that CTA the tile is the last unit of its
+                    // range, so it gets here last in time, while every other contributor handles its share as the
+                    // first unit of its range (or as its only one), stores it and counts itself in without ever
+                    // waiting.  The finisher keeps its own share in tensor memory and waits (bounded) for the
+                    // others; they run at the same time on other SMs and depend on nobody, so the wait is short:
+                    // the store and count of a contributor that ended together with the finisher.
+                    if (et == 0) {
+                        int fl = 0;
+                        if (cta == c_first) {
+                            fl = 1;
+                            uint32_t spin = 0;
+                            while (ld_acquire_gpu(p.counters + tile) != c_last - c_first) {
+                                if (++spin >= SPIN_LIMIT) { *abort_flag = 1; atomicCAS(p.status, DEV_OK, DEV_TIMEOUT_GRID); break; }
+                                __nanosleep(spin > 64 ? 64 : 20);
+                            }
+                        }
+                        sm->last_flag = fl;
+                    }
                     epi_all();
                     finish = sm->last_flag != 0;
                     epi_all();
@@ -253,10 +268,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                         // count this arrival: the barrier orders every thread's stores before thread 0's
                         // release, and the release is cumulative over them
                         epi_all();
-                        if (et == 0) sm->last_flag = (atom_add_acq_rel_gpu(p.counters + tile, 1) == c_last - c_first) ? 1 : 0;
-                        epi_all();
-                        finish = sm->last_flag != 0;
-                        epi_all();
+                        if (et == 0) atom_add_acq_rel_gpu(p.counters + tile, 1);
                     }
                 }
                 if (finish) {
