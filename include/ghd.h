@@ -59,7 +59,11 @@ typedef enum ghd_option {
     GHD_OPT_NO_PDL = 6,       /* 1 = launch every kernel fully serialised (no programmatic
                                  dependent launch overlap between consecutive kernels)        */
     GHD_OPT_GEMM_STAGES = 7,  /* pipeline stages of the tcgen05 GEMM (0 = automatic)          */
-    GHD_OPT_GEMM_EPI = 8      /* epilogue warp groups of the tcgen05 GEMM: 0 auto, 1, 2        */
+    GHD_OPT_GEMM_EPI = 8,     /* epilogue warp groups of the tcgen05 GEMM: 0 auto, 1, 2        */
+    GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
+                                 Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
+                                 nobody sees them (default); 1 = per-query list of visible nodes (the
+                                 COO index): each query gathers only the keys it sees                */
 } ghd_option;
 
 /* LLaMA-style decoder (paper Sec. IV-A: Vicuna-7B / LLaMA-7B): RMSNorm, rotary
@@ -103,12 +107,19 @@ typedef struct ghd_kv_layer {
  *   mask[i * n_words + w] bit b  = 1 iff new node (64 w + b) is visible to node i
  *                                  (ancestor or i itself), LSB first;
  *   depth[i] = edges from the root, pos[i] = kv_len + depth[i] (position id);
- *   rope[i * d_head + 2 t], [.. + 2 t + 1] = cos, sin of pos[i] * theta^(-2 t / d_head). */
+ *   rope[i * d_head + 2 t], [.. + 2 t + 1] = cos, sin of pos[i] * theta^(-2 t / d_head).
+ * Optional (both NULL, or both given): the same visibility as a sparse index in coordinate order
+ * (Sec. III-B-3: the index of the token pairs to verify is generated before the inference),
+ *   coo_ptr: int32 [max_nodes + 1], coo_col: int32 [max_nodes * (max_nodes + 1) / 2];
+ *   the visible new nodes of query i are coo_col[coo_ptr[i] .. coo_ptr[i + 1]), ascending; nnz = coo_ptr[n].
+ * GHD_OPT_ATTN_SPARSE = 1 needs it. */
 typedef struct ghd_tree {
     int32_t n, kv_len, n_words, has_parent;
     uint64_t *mask;
     int32_t *parent, *depth, *pos;
     float *rope;
+    int32_t *coo_ptr, *coo_col;
+    int32_t nnz;
 } ghd_tree;
 
 /* dev struct written by ghd_accept.  nodes[0..n_matched] is the accepted root
@@ -142,7 +153,8 @@ typedef enum ghd_path {
     GHD_PATH_GEMM_TILE = 0,   /* tcgen05 projection, stream-K over 128-row tiles      */
     GHD_PATH_GEMM_SIMT = 1,   /* CUDA-core projection                                 */
     GHD_PATH_ATTN_TC = 2,     /* tcgen05 tree attention                               */
-    GHD_PATH_ATTN_SIMT = 3    /* CUDA-core tree attention                             */
+    GHD_PATH_ATTN_SIMT = 3,   /* CUDA-core tree attention                             */
+    GHD_PATH_ATTN_COO = 4     /* sparse part gathered from the coordinate index        */
 } ghd_path;
 int64_t ghd_path_count(const ghd_ctx *ctx, int32_t path);
 
@@ -174,6 +186,12 @@ ghd_status ghd_verify_layer(ghd_ctx *ctx, const ghd_layer_weights *w, ghd_kv_lay
  * the logits live only in the workspace); argmax_dev: int32 [n]. */
 ghd_status ghd_verify_step(ghd_ctx *ctx, const ghd_model_weights *w, ghd_kv_layer *kv, const ghd_tree *tree,
                            const int32_t *tokens_dev, float *logits_dev, int32_t *argmax_dev);
+
+/* The hidden states the last ghd_verify_step of this context produced: the output of the last layer
+ * (Sec. II-B: what the layer stack hands to the final norm and the lm_head), float, before the final
+ * RMSNorm.  Copies rows [0, n) of width d_model to dst_dev (dev float [n][d_model]) on the context's stream.
+ * GHD_EINVAL on a null pointer or n outside [1, max_nodes]; GHD_ENOSPACE without a workspace. */
+ghd_status ghd_copy_hidden(ghd_ctx *ctx, int32_t n, float *dst_dev);
 
 /* Greedy acceptance (Sec. II-C: fall back to the longest validated prefix): node
  * c is valid iff every edge (p -> c') on its root path has tokens[c'] == argmax[p];

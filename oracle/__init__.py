@@ -118,6 +118,22 @@ def tree_build(parent, kv_len: int):
     return vis, depth, pos
 
 
+def coo_index(vis):
+    """The visibility among the drafted nodes as a sparse index in coordinate order (paper Sec. III-B-3: the
+    index of the token pairs to verify is written down before the inference): every (query i, node j) with
+    vis[i][j] set, sorted by i then j, plus the row starts.  -> (ptr int32 [n + 1], cols int32 [nnz]).
+    Plain restatement: a scan of the matrix, one pair at a time."""
+    vis = np.asarray(vis)
+    n = vis.shape[0]
+    ptr, cols = [0], []
+    for i in range(n):
+        for j in range(n):
+            if vis[i][j]:
+                cols.append(j)
+        ptr.append(len(cols))
+    return np.asarray(ptr, dtype=np.int32), np.asarray(cols, dtype=np.int32)
+
+
 def rmsnorm(x, g, eps: float):
     x, g = _f64(x), _stored(g)
     out = np.empty_like(x)

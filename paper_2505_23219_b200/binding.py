@@ -17,19 +17,19 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_copy_hidden", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
     "MedusaWeights", "GHD_MAX_TOPK",
-    "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT",
+    "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_ATTN_COO",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
 GHD_MAX_TOPK = 16
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
-OPT_GEMM_STAGES, OPT_GEMM_EPI = 7, 8
-PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT = 0, 1, 2, 3
+OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE = 7, 8, 9
+PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_ATTN_COO = 0, 1, 2, 3, 4
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
 
@@ -39,7 +39,7 @@ EXPORTS = [
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
     "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit",
-    "ghd_medusa_draft", "ghd_tree_fill_tokens",
+    "ghd_medusa_draft", "ghd_tree_fill_tokens", "ghd_copy_hidden",
 ]
 
 
@@ -76,7 +76,7 @@ class _Kv(C.Structure):
 class _Tree(C.Structure):
     _fields_ = [("n", C.c_int32), ("kv_len", C.c_int32), ("n_words", C.c_int32), ("has_parent", C.c_int32),
                 ("mask", C.c_void_p), ("parent", C.c_void_p), ("depth", C.c_void_p), ("pos", C.c_void_p),
-                ("rope", C.c_void_p)]
+                ("rope", C.c_void_p), ("coo_ptr", C.c_void_p), ("coo_col", C.c_void_p), ("nnz", C.c_int32)]
 
 
 _LIB = None
@@ -105,6 +105,7 @@ def load_library(path: str | Path | None = None):
         "ghd_verify_layer": ([vp, C.POINTER(_LayerW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp], C.c_int),
         "ghd_verify_step": ([vp, C.POINTER(_ModelW), C.POINTER(_Kv), C.POINTER(_Tree), vp, vp, vp], C.c_int),
         "ghd_accept": ([vp, C.POINTER(_Tree), vp, vp, vp], C.c_int),
+        "ghd_copy_hidden": ([vp, i32, vp], C.c_int),
         "ghd_kv_commit": ([vp, C.POINTER(_Kv), i32, i32, vp], C.c_int),
         "ghd_medusa_draft": ([vp, C.POINTER(_MedusaW), vp, vp, vp, vp], C.c_int),
         "ghd_tree_fill_tokens": ([vp, vp, vp, vp, vp, i32, vp], C.c_int),
@@ -186,12 +187,20 @@ class Tree:
         self.depth = torch.zeros(n, dtype=torch.int32, device=dev)
         self.pos = torch.zeros(n, dtype=torch.int32, device=dev)
         self.rope = torch.zeros(n * ctx.cfg.c.d_head, dtype=torch.float32, device=dev)
+        self.coo_ptr = torch.zeros(n + 1, dtype=torch.int32, device=dev)
+        self.coo_col = torch.zeros(n * (n + 1) // 2, dtype=torch.int32, device=dev)
         self.c = _Tree(0, 0, 0, 0, _ptr(self.mask), _ptr(self.parent), _ptr(self.depth), _ptr(self.pos),
-                       _ptr(self.rope))
+                       _ptr(self.rope), _ptr(self.coo_ptr), _ptr(self.coo_col), 0)
 
     @property
     def n(self):
         return self.c.n
+
+    def coo(self):
+        """-> (row pointers int32 [n + 1], visible node ids int32 [nnz]) on the host."""
+        n = self.c.n
+        ptr = self.coo_ptr[: n + 1].cpu().numpy()
+        return ptr, self.coo_col[: int(ptr[n])].cpu().numpy()
 
     def mask_words(self) -> np.ndarray:
         """mask as uint64 [n][n_words] on the host."""
@@ -301,6 +310,14 @@ def ghd_verify_step(ctx: Ctx, w: ModelWeights, kvs, tree: Tree, tokens, logits=N
     ctx._check(ctx.lib.ghd_verify_step(ctx.handle, C.byref(w.c), arr, C.byref(tree.c), tokens.data_ptr(),
                                        _ptr(logits), argmax.data_ptr()))
     return logits, argmax
+
+
+def ghd_copy_hidden(ctx: Ctx, n: int, out=None):
+    """-> float32 device tensor [n][d_model]: the last layer's output of the last ghd_verify_step (before the final norm)."""
+    if out is None:
+        out = torch.empty((n, ctx.cfg.c.d_model), dtype=torch.float32, device=ctx.device)
+    ctx._check(ctx.lib.ghd_copy_hidden(ctx.handle, n, out.data_ptr()))
+    return out
 
 
 def ghd_accept(ctx: Ctx, tree: Tree, tokens, argmax, out=None):

@@ -32,7 +32,7 @@ template <> __device__ __forceinline__ __half st_cvt<__half>(float v) { return _
 template <typename T, int DH>
 __global__ void __launch_bounds__(QB * 32)
 k_attn_simt(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
-            const uint64_t* __restrict__ mask, int n_words, int n, int heads, int kv_len, int max_kv,
+            const uint64_t* __restrict__ mask, int n_words, int n, int n_new, int heads, int kv_len, int max_kv,
             int chunk, float* __restrict__ part_o, float* __restrict__ part_ml, int max_nodes) {
     constexpr int R = DH / 32;
     __shared__ float sq[QB][DH];
@@ -43,7 +43,7 @@ k_attn_simt(const T* __restrict__ q, const T* __restrict__ kc, const T* __restri
     const int i = blockIdx.x * QB + warp;
     const bool live = i < n;
     const int d = heads * DH;
-    const int kt = kv_len + n;
+    const int kt = kv_len + n_new;                         // n_new = n, or 0 when the new rows are handled elsewhere
     const int j_begin = split * chunk, j_end = min(kt, j_begin + chunk);
     const float scale = rsqrtf((float)DH);
     for (int c = lane; c < DH; c += 32) sq[warp][c] = live ? ld_f32<T>(q + (size_t)i * d + h * DH + c) * scale : 0.f;
@@ -102,6 +102,79 @@ k_attn_simt(const T* __restrict__ q, const T* __restrict__ kc, const T* __restri
             pm[0] = m;
             pm[1] = l;
         }
+    }
+}
+
+// Sparse part of the tree attention from a coordinate index (paper Sec. III-B-3: the visible (query, key)
+// pairs are listed before the inference; Q K^T touches one row of Q and one row of K per pair, A V adds
+// A[i][j] * V[j] into row i of O, which stays in registers until the row's pairs are exhausted).  One warp per
+// (query, head): lane t holds DH / 32 consecutive columns of q, of the output row and of every K / V row it
+// reads (a row is one coalesced request of the warp); a query with depth + 1 visible nodes reads exactly that
+// many rows, whatever the size of the tree.  Leaves the un-normalised (o, max, sum) of the new-row part.
+constexpr int COO_WARPS = 4;
+
+// R consecutive elements (R = 2 or 4, the address R-element aligned) in one request, widened to float.
+template <typename T, int R>
+__device__ __forceinline__ void ld_row_piece(const T* p, float (&v)[R]) {
+    if constexpr (sizeof(T) == 4) {
+        if constexpr (R == 4) { const float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+        else { const float2 t = *reinterpret_cast<const float2*>(p); v[0] = t.x; v[1] = t.y; }
+    } else {
+        if constexpr (R == 4) {
+            const uint2 t = *reinterpret_cast<const uint2*>(p);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&t.y));
+            v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+        } else {
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(p));
+            v[0] = a.x; v[1] = a.y;
+        }
+    }
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(COO_WARPS * 32)
+k_attn_coo(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc, const int32_t* __restrict__ coo_ptr,
+           const int32_t* __restrict__ coo_col, int n, int heads, int kv_len, int max_kv,
+           float* __restrict__ part_o, float* __restrict__ part_ml) {
+    constexpr int R = DH / 32;
+    pdl_wait();
+    pdl_trigger();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * COO_WARPS + warp, h = blockIdx.y;
+    if (i >= n) return;
+    const int d = heads * DH;
+    const float scale = rsqrtf((float)DH);
+    float qv[R], o[R];
+    ld_row_piece<T, R>(q + (size_t)i * d + h * DH + lane * R, qv);
+#pragma unroll
+    for (int r = 0; r < R; ++r) { qv[r] *= scale; o[r] = 0.f; }
+    const T* kbase = kc + ((size_t)h * max_kv + kv_len) * DH + lane * R;
+    const T* vbase = vc + ((size_t)h * max_kv + kv_len) * DH + lane * R;
+    float m = -INFINITY, l = 0.f;
+    const int e0 = coo_ptr[i], e1 = coo_ptr[i + 1];
+    for (int e = e0; e < e1; ++e) {
+        const int j = coo_col[e];
+        float kr[R], vr[R], s = 0.f;
+        ld_row_piece<T, R>(kbase + (size_t)j * DH, kr);
+        ld_row_piece<T, R>(vbase + (size_t)j * DH, vr);
+#pragma unroll
+        for (int r = 0; r < R; ++r) s = fmaf(qv[r], kr[r], s);
+        for (int sh = 16; sh > 0; sh >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sh);
+        const float m_new = fmaxf(m, s);
+        const float corr = (m == -INFINITY) ? 0.f : expf(m - m_new);
+        const float pj = expf(s - m_new);
+        l = l * corr + pj;
+#pragma unroll
+        for (int r = 0; r < R; ++r) o[r] = fmaf(pj, vr[r], o[r] * corr);
+        m = m_new;
+    }
+    float* po = part_o + (size_t)i * d + h * DH + lane * R;
+#pragma unroll
+    for (int r = 0; r < R; ++r) po[r] = o[r];
+    if (lane == 0) {
+        float* pm = part_ml + ((size_t)i * heads + h) * 2;
+        pm[0] = m;
+        pm[1] = l;
     }
 }
 
@@ -188,22 +261,24 @@ int attn_auto_splits(const ghd_ctx* c, int n, int kv_total) {
     return s < 1 ? 1 : s;
 }
 
-void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
+void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo) {
     const ghd_model_cfg& m = c->cfg;
-    const int kt = t->kv_len + t->n;
+    const int n_new = coo ? 0 : t->n;
+    const int kt = t->kv_len + n_new;
     int splits = c->opt_attn_splits > 0 ? c->opt_attn_splits : attn_auto_splits(c, t->n, kt);
-    if (splits > c->max_splits) splits = c->max_splits;
+    if (splits > c->max_splits - (coo ? 1 : 0)) splits = c->max_splits - (coo ? 1 : 0);
     int chunk = (kt + splits - 1) / splits;
     chunk = ((chunk + TK - 1) / TK) * TK;
     dim3 grid((t->n + QB - 1) / QB, m.n_heads, splits);
 #define GHD_ATTN(T, DH)                                                                                          \
     k_attn_simt<T, DH><<<grid, QB * 32, 0, c->cur>>>((const T*)q, (const T*)kv->k, (const T*)kv->v, t->mask,  \
-                                                        t->n_words, t->n, m.n_heads, t->kv_len, m.max_kv_len,    \
+                                                        t->n_words, t->n, n_new, m.n_heads, t->kv_len, m.max_kv_len, \
                                                         chunk, c->att_o, c->att_ml, m.max_nodes)
     if (m.dtype == GHD_F32) { if (m.d_head == 64) GHD_ATTN(float, 64); else GHD_ATTN(float, 128); }
     else { if (m.d_head == 64) GHD_ATTN(__half, 64); else GHD_ATTN(__half, 128); }
 #undef GHD_ATTN
     c->launches++;
+    if (coo) { launch_attn_coo(c, q, kv, t, splits); ++splits; }      // the sparse part as one more partial
     dim3 cgrid(t->n, m.n_heads);
     if (m.dtype == GHD_F32)
         k_attn_combine<float><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (float*)out, splits, m.n_heads,
@@ -212,6 +287,18 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
         k_attn_combine<__half><<<cgrid, m.d_head, 0, c->cur>>>(c->att_o, c->att_ml, (__half*)out, splits, m.n_heads,
                                                                   m.d_head, m.max_nodes);
     c->launches++;
+}
+
+void launch_attn_coo(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, int slot) {
+    const ghd_model_cfg& m = c->cfg;
+    dim3 grid((t->n + COO_WARPS - 1) / COO_WARPS, m.n_heads);
+#define GHD_COO(T, DH)                                                                                              \
+    launch_k(c, true, k_attn_coo<T, DH>, grid, dim3(COO_WARPS * 32), 0, (const T*)q, (const T*)kv->k, (const T*)kv->v,   \
+             (const int32_t*)t->coo_ptr, (const int32_t*)t->coo_col, t->n, m.n_heads, t->kv_len, m.max_kv_len,      \
+             c->att_o + (size_t)slot * m.max_nodes * m.d_model, c->att_ml + (size_t)slot * m.max_nodes * m.n_heads * 2)
+    if (m.dtype == GHD_F32) { if (m.d_head == 64) GHD_COO(float, 64); else GHD_COO(float, 128); }
+    else { if (m.d_head == 64) GHD_COO(__half, 64); else GHD_COO(__half, 128); }
+#undef GHD_COO
 }
 
 void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n) {
@@ -324,7 +411,7 @@ extern "C" ghd_status ghd_tree_attention_static(void* cuda_stream, int32_t dtype
     const int n_words = (n + 63) / 64;
 #define GHD_ATTN_ST(T, DH)                                                                                  \
     k_attn_simt<T, DH><<<grid, QB * 32, 0, stream>>>((const T*)q, (const T*)k_cache, (const T*)v_cache,      \
-                                                     mask_dev, n_words, n, n_heads, kv_len, max_kv_len,      \
+                                                     mask_dev, n_words, n, n, n_heads, kv_len, max_kv_len,   \
                                                      chunk, part_o, part_ml, ST_MAX_NODES)
     if (dtype == GHD_F32) { if (d_head == 64) GHD_ATTN_ST(float, 64); else GHD_ATTN_ST(float, 128); }
     else { if (d_head == 64) GHD_ATTN_ST(__half, 64); else GHD_ATTN_ST(__half, 128); }

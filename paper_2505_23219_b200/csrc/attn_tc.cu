@@ -44,6 +44,7 @@ constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 
 struct AttnParams {
     int n, heads, kv_len, max_nodes, splits, n_words;
+    int cache_only;            // 1: the new rows are somebody else's (the coordinate-index kernel): no node groups here
     const uint64_t* mask;
     float* part_o;
     float* part_ml;
@@ -146,7 +147,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     uint32_t cand = 0;
 #pragma unroll
     for (int w = 0; w < MAX_UNITS_WORDS; ++w)
-        if (w < p.n_words && p.splits - 1 - (w % p.splits) == split) cand |= 1u << w;
+        if (!p.cache_only && w < p.n_words && p.splits - 1 - (w % p.splits) == split) cand |= 1u << w;
     // body(i, key0, w): unit number, first key row, node group (-1 for a cache tile); false stops the walk
     auto walk = [&](auto&& body) -> int {
         int i = 0;
@@ -571,7 +572,7 @@ bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t) {
     return c->cfg.dtype == GHD_F16 && (c->cfg.d_head == 64 || c->cfg.d_head == 128) && t->n >= 1;
 }
 
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo) {
     const ghd_model_cfg& m = c->cfg;
     const int n = t->n, H = m.n_heads, dh = m.d_head, d = m.d_model;
     const int kt = t->kv_len + n;
@@ -588,16 +589,17 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         return GHD_ECUDA;
     }
     const int mtiles = (n + QM - 1) / QM;
-    const int units = (t->kv_len + BN - 1) / BN + t->n_words;
+    const int units = (t->kv_len + BN - 1) / BN + (coo ? 0 : t->n_words);
     int splits = c->opt_attn_splits;
     if (splits <= 0) {
         splits = c->sm_count / (H * mtiles);
         const int by_len = (units + 1) / 2;              // at least two units per split
         if (splits > by_len) splits = by_len;
     }
-    if (splits > c->max_splits) splits = c->max_splits;
+    if (splits > c->max_splits - (coo ? 1 : 0)) splits = c->max_splits - (coo ? 1 : 0);    // the index kernel's partial takes a slot
     if (splits < 1) splits = 1;
     AttnParams p{};
+    p.cache_only = coo ? 1 : 0;
     p.n = n; p.heads = H; p.kv_len = t->kv_len; p.max_nodes = m.max_nodes; p.splits = splits; p.n_words = t->n_words;
     p.mask = t->mask; p.part_o = c->att_o; p.part_ml = c->att_ml; p.status = c->status;
     p.scale = 1.0f / sqrtf((float)dh);
@@ -621,7 +623,8 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         if (pair) launch_k(c, true, k_attn_tc<128, true>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
         else launch_k(c, true, k_attn_tc<128, false>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
     }
-    launch_attn_combine(c, out, splits, n);
+    if (coo) launch_attn_coo(c, q, kv, t, splits);       // the sparse part as one more partial, slot `splits`
+    launch_attn_combine(c, out, splits + (coo ? 1 : 0), n);
     return GHD_OK;
 }
 

@@ -100,10 +100,13 @@ static ghd_status project_residual(ghd_ctx* c, const void* x, const void* w, int
 
 static ghd_status attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out) {
     const bool tc_ok = attn_tc_supported(c, t);
+    const bool coo = c->opt_attn_sparse == 1;
+    if (coo && (!t->coo_ptr || !t->coo_col)) return fail(c, GHD_EINVAL, "attention: the tree carries no coordinate index");
     if (c->opt_attn_path == 2 && !tc_ok) return fail(c, GHD_EUNSUPPORTED, "tcgen05 attention does not take this type/shape");
-    if (tc_ok && c->opt_attn_path != 1) { c->path_count[GHD_PATH_ATTN_TC]++; return launch_attn_tc(c, q, kv, t, out); }
+    if (coo) c->path_count[GHD_PATH_ATTN_COO]++;
+    if (tc_ok && c->opt_attn_path != 1) { c->path_count[GHD_PATH_ATTN_TC]++; return launch_attn_tc(c, q, kv, t, out, coo); }
     c->path_count[GHD_PATH_ATTN_SIMT]++;
-    launch_attn_simt(c, q, kv, t, out);
+    launch_attn_simt(c, q, kv, t, out, coo);
     return GHD_OK;
 }
 
@@ -173,7 +176,7 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
@@ -226,6 +229,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
         case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
         case GHD_OPT_GEMM_STAGES: if (value == 1 || value > 10) return GHD_EINVAL; c->opt_gemm_stages = value; break;
+        case GHD_OPT_ATTN_SPARSE: if (value > 1) return GHD_EINVAL; c->opt_attn_sparse = value; break;
         case GHD_OPT_GEMM_EPI: if (value > 2) return GHD_EINVAL; c->opt_gemm_epi = value; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
         default: return GHD_EINVAL;
@@ -236,6 +240,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
 static ghd_status tree_common(ghd_ctx* c, int32_t n, int32_t kv_len, ghd_tree* tree) {
     if (!c || !tree) return GHD_EINVAL;
     if (!tree->mask || !tree->parent || !tree->depth || !tree->pos || !tree->rope) return fail(c, GHD_EINVAL, "tree: null buffer");
+    if ((tree->coo_ptr == nullptr) != (tree->coo_col == nullptr)) return fail(c, GHD_EINVAL, "tree: give both index buffers or neither");
     if (n < 1 || n > c->cfg.max_nodes) return fail(c, GHD_ETREE, "tree: n outside [1, max_nodes]");
     if (kv_len < 0) return fail(c, GHD_EINVAL, "tree: negative kv_len");
     if ((int64_t)kv_len + n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: kv_len + n > max_kv_len");
@@ -276,7 +281,7 @@ ghd_status ghd_tree_from_mask(ghd_ctx* c, const uint64_t* mask_host, const int32
     cudaMemcpyAsync(tree->mask, mask_host, sizeof(uint64_t) * n * W, cudaMemcpyHostToDevice, c->stream);
     if (depth_host) cudaMemcpyAsync(tree->depth, depth_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream);
     if (parent_host) cudaMemcpyAsync(tree->parent, parent_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream);
-    launch_tree_from_mask(c, tree, depth_host != nullptr);
+    launch_tree_from_mask(c, tree, depth_host != nullptr, mask_host);
     return check_cuda(c, "tree_from_mask");
 }
 
@@ -323,9 +328,9 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     std::vector<uint64_t> key;
     auto push = [&](const void* p) { key.push_back((uint64_t)(uintptr_t)p); };
     push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
-    push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope);
+    push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope); push(tree->coo_ptr); push(tree->coo_col);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
-    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi})
+    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse})
         key.push_back((uint64_t)(uint32_t)o);       // every option that changes what is enqueued
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
@@ -359,6 +364,14 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     if (c->graphs->size() >= 8) { cudaGraphExecDestroy(c->graphs->front()->exec); delete c->graphs->front(); c->graphs->erase(c->graphs->begin()); }
     c->graphs->push_back(g);
     if (cudaGraphLaunch(exec, c->stream) != cudaSuccess) return check_cuda(c, "graph launch");
+    return GHD_OK;
+}
+
+ghd_status ghd_copy_hidden(ghd_ctx* c, int32_t n, float* dst_dev) {
+    if (!c || !dst_dev || n < 1 || n > c->cfg.max_nodes) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (cudaMemcpyAsync(dst_dev, c->xres, sizeof(float) * (size_t)n * c->cfg.d_model, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+        return check_cuda(c, "copy_hidden");
     return GHD_OK;
 }
 

@@ -68,7 +68,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -148,8 +148,8 @@ inline cudaError_t launch_k(ghd_ctx* c, bool pdl, void (*kernel)(KArgs...), dim3
 size_t carve_workspace(ghd_ctx* c, char* base);   // returns bytes needed; assigns pointers when base != nullptr
 
 // kernels_small.cu
-void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t);
-void launch_tree_from_mask(ghd_ctx* c, const ghd_tree* t, bool have_depth);   // mask/depth already copied
+void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, ghd_tree* t);
+void launch_tree_from_mask(ghd_ctx* c, ghd_tree* t, bool have_depth, const uint64_t* mask_host);   // mask/depth already copied
 void launch_load_x(ghd_ctx* c, const void* x_in, int n);     // T [n][d] -> xres
 void launch_store_x(ghd_ctx* c, void* x_out, int n);         // xres -> T [n][d]
 void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n);
@@ -172,7 +172,10 @@ void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_l
 void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, float* y);
 
 // attn_simt.cu : split-KV tree attention + combine
-void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
+void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo);
+// The sparse part from the coordinate index: every query gathers the new keys/values it sees; the result
+// goes to partial slot `slot` of att_o / att_ml (natural-log maxima), to be merged with the cache splits.
+void launch_attn_coo(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, int slot);
 int attn_auto_splits(const ghd_ctx* c, int n, int kv_total);
 
 void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n);   // merges att_o / att_ml into out
@@ -180,7 +183,8 @@ void launch_attn_combine(ghd_ctx* c, void* out, int splits, int n);   // merges 
 // attn_tc.cu : tcgen05 / TMA tree attention (GHD_F16 only)
 bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t);
 // the split partials go to att_o / att_ml and a second kernel merges them into `out`
-ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out);
+// coo: the new rows are handled by launch_attn_coo (one more partial), this kernel takes the cache only
+ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo);
 
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);

@@ -16,6 +16,8 @@ template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return
 
 // ---------------------------------------------------------------- tree build
 struct ParentArg { int16_t p[GHD_MAX_NODES]; };
+// Row starts of the coordinate index (nnz <= 256 * 257 / 2 fits 16 bits), worked out on the host.
+struct CooPtrArg { uint16_t ptr[GHD_MAX_NODES + 1]; };
 
 // Block b takes nodes 8b .. 8b+7: one thread per node walks to the root, setting one mask bit per
 // ancestor; then the block fills those nodes' rows of the rotary table.  The table is computed in
@@ -23,8 +25,9 @@ struct ParentArg { int16_t p[GHD_MAX_NODES]; };
 // the slow part (pow and sincos in double), hence several blocks.
 constexpr int TREE_NODES_PER_BLOCK = 8;
 
-__global__ void k_tree_build(ParentArg pa, int n, int n_words, int kv_len, int d_head, double theta,
-                             uint64_t* mask, int32_t* parent, int32_t* depth, int32_t* pos, float* rope) {
+__global__ void k_tree_build(ParentArg pa, CooPtrArg cp, int n, int n_words, int kv_len, int d_head, double theta,
+                             uint64_t* mask, int32_t* parent, int32_t* depth, int32_t* pos, float* rope,
+                             int32_t* coo_ptr, int32_t* coo_col) {
     __shared__ int spos[TREE_NODES_PER_BLOCK];
     const int first = blockIdx.x * TREE_NODES_PER_BLOCK;
     if (threadIdx.x < TREE_NODES_PER_BLOCK) {
@@ -35,6 +38,13 @@ __global__ void k_tree_build(ParentArg pa, int n, int n_words, int kv_len, int d
             int steps = 0;
             for (int a = i; a >= 0 && steps <= n; a = pa.p[a]) { row[a >> 6] |= 1ull << (a & 63); ++steps; }
             for (int w = 0; w < n_words; ++w) mask[i * n_words + w] = row[w];
+            if (coo_ptr) {
+                // the same walk again, filling the row's list from its end: ancestors come out in descending order
+                coo_ptr[i] = cp.ptr[i];
+                if (i == n - 1) coo_ptr[n] = cp.ptr[n];
+                int at = cp.ptr[i + 1], left = steps;
+                for (int a = i; a >= 0 && left > 0 && at > cp.ptr[i]; a = pa.p[a], --left) coo_col[--at] = a;
+            }
             parent[i] = pa.p[i];
             depth[i] = steps - 1;
             p = kv_len + steps - 1;
@@ -56,9 +66,16 @@ __global__ void k_tree_build(ParentArg pa, int n, int n_words, int kv_len, int d
 }
 
 // Explicit-mask variant: mask (and optionally depth, parent) were copied in.
-__global__ void k_tree_from_mask(int n, int n_words, int kv_len, int d_head, double theta, int have_depth,
-                                 const uint64_t* mask, int32_t* depth, int32_t* pos, float* rope) {
+__global__ void k_tree_from_mask(CooPtrArg cp, int n, int n_words, int kv_len, int d_head, double theta, int have_depth,
+                                 const uint64_t* mask, int32_t* depth, int32_t* pos, float* rope, int32_t* coo_ptr, int32_t* coo_col) {
     const int i = threadIdx.x;
+    if (i < n && coo_ptr) {
+        coo_ptr[i] = cp.ptr[i];
+        if (i == n - 1) coo_ptr[n] = cp.ptr[n];
+        int at = cp.ptr[i];
+        for (int w = 0; w < n_words; ++w)
+            for (uint64_t bits = mask[i * n_words + w]; bits && at < cp.ptr[i + 1]; bits &= bits - 1) coo_col[at++] = 64 * w + __ffsll((long long)bits) - 1;
+    }
     if (i < n) {
         int dep;
         if (have_depth) dep = depth[i];
@@ -82,19 +99,40 @@ __global__ void k_tree_from_mask(int n, int n_words, int kv_len, int d_head, dou
     }
 }
 
-void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, const ghd_tree* t) {
+void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, ghd_tree* t) {
     ParentArg pa;
-    for (int i = 0; i < GHD_MAX_NODES; ++i) pa.p[i] = (int16_t)(i < t->n ? parent_host[i] : -1);
-    k_tree_build<<<(t->n + TREE_NODES_PER_BLOCK - 1) / TREE_NODES_PER_BLOCK, 256, 0, c->cur>>>(pa, t->n, t->n_words, t->kv_len, c->cfg.d_head,
+    CooPtrArg cp;
+    int depth[GHD_MAX_NODES];
+    cp.ptr[0] = 0;
+    for (int i = 0; i < GHD_MAX_NODES; ++i) {
+        pa.p[i] = (int16_t)(i < t->n ? parent_host[i] : -1);
+        if (i < t->n) {                                   // row i lists node i and its ancestors: depth + 1 entries
+            depth[i] = i == 0 ? 0 : depth[parent_host[i]] + 1;
+            cp.ptr[i + 1] = (uint16_t)(cp.ptr[i] + depth[i] + 1);
+        } else {
+            cp.ptr[i + 1] = cp.ptr[i];
+        }
+    }
+    t->nnz = cp.ptr[t->n];
+    k_tree_build<<<(t->n + TREE_NODES_PER_BLOCK - 1) / TREE_NODES_PER_BLOCK, 256, 0, c->cur>>>(pa, cp, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                      (double)c->cfg.rope_theta, t->mask, t->parent, t->depth,
-                                                     t->pos, t->rope);
+                                                     t->pos, t->rope, t->coo_ptr, t->coo_col);
     c->launches++;
 }
 
-void launch_tree_from_mask(ghd_ctx* c, const ghd_tree* t, bool have_depth) {
-    k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->cur>>>(t->n, t->n_words, t->kv_len, c->cfg.d_head,
+void launch_tree_from_mask(ghd_ctx* c, ghd_tree* t, bool have_depth, const uint64_t* mask_host) {
+    CooPtrArg cp;
+    cp.ptr[0] = 0;
+    for (int i = 0; i < GHD_MAX_NODES; ++i) {
+        int bits = 0;
+        if (i < t->n)
+            for (int w = 0; w < t->n_words; ++w) bits += __builtin_popcountll(mask_host[(size_t)i * t->n_words + w]);
+        cp.ptr[i + 1] = (uint16_t)(cp.ptr[i] + bits);
+    }
+    t->nnz = cp.ptr[t->n];
+    k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->cur>>>(cp, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                          (double)c->cfg.rope_theta, have_depth ? 1 : 0, t->mask,
-                                                         t->depth, t->pos, t->rope);
+                                                         t->depth, t->pos, t->rope, t->coo_ptr, t->coo_col);
     c->launches++;
 }
 

@@ -24,7 +24,8 @@ CONFIG_ID = 3
 KV_LEN = 2048
 N = 64
 PLANT = 3
-SAMPLES_PER_ROW = 12
+SAMPLES_PER_ROW = 512      # logit columns stored per node, the oracle's top 8 among them
+HIDDEN_COLS = 64           # columns of the last layer's output stored per node
 
 
 def main():
@@ -64,7 +65,7 @@ def main():
         assert len(sib) == len(set(sib)), "duplicate sibling tokens after planting"
 
     vis, depth, pos = oracle.tree_build(parent, KV_LEN)
-    logits, amax = oracle.step(shape, head, layers, fresh(), KV_LEN, vis, pos, tokens)
+    logits, amax, hidden = oracle.step(shape, head, layers, fresh(), KV_LEN, vis, pos, tokens, want_hidden=True)
     print(f"full step done ({time.time() - t0:.0f}s)", flush=True)
     m, nodes, emitted = oracle.accept(parent, tokens, amax)
     assert m == PLANT and list(nodes) == chain, (m, list(nodes), chain)
@@ -74,8 +75,12 @@ def main():
     rng = wl.Rng(wl.BASE_SEED + 1000 * CONFIG_ID + 701)
     samples = []
     for i in range(N):
-        cols = sorted({int(amax[i])} | {rng.below(shape.vocab) for _ in range(SAMPLES_PER_ROW)})
-        samples.append({"node": i, "cols": cols, "values": [float(f"{logits[i, c]:.12e}") for c in cols]})
+        cols = {int(c) for c in np.argsort(logits[i])[-8:]}
+        while len(cols) < SAMPLES_PER_ROW:
+            cols.add(rng.below(shape.vocab))
+        cols = sorted(cols)
+        samples.append({"node": i, "cols": cols, "values": [float(f"{logits[i, c]:.9e}") for c in cols]})
+    hcols = sorted({rng.below(shape.d_model) for _ in range(4 * HIDDEN_COLS)})[:HIDDEN_COLS]
     out = {
         "source": "tests/golden/make_c3_fixture.py (CPU oracle only)",
         "config": {"shape": shape.name, "config_id": CONFIG_ID, "kv_len": KV_LEN, "n": N, "tree": "medusa_tree(64)"},
@@ -90,9 +95,12 @@ def main():
         "row_margins": [float(f"{v:.6e}") for v in margins],
         "runner_up": [int(np.argsort(logits[i])[-2]) for i in range(N)],
         "logit_samples": samples,
+        "hidden_abs_max": float(np.abs(hidden).max()),
+        "hidden_cols": hcols,
+        "hidden_samples": [[float(f"{hidden[i, c]:.9e}") for c in hcols] for i in range(N)],
     }
     path = Path(__file__).resolve().parent / "c3_step_llama7b.json"
-    path.write_text(json.dumps(out, indent=1))
+    path.write_text(json.dumps(out, separators=(",", ":")).replace("},{", "},\n{"))
     print(f"wrote {path} ({time.time() - t0:.0f}s); min top-2 margin {margins.min():.4f}", flush=True)
 
 

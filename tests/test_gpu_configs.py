@@ -22,9 +22,10 @@ def ghd():
     return g
 
 
-def _layer_parity(ghd, shape, w, gw, config_id, n, L, parent=None, vis=None, depth=None):
+def _layer_parity(ghd, shape, w, gw, config_id, n, L, parent=None, vis=None, depth=None, sparse=0):
     Lmax = L + n
     ctx = ghd.ghd_create(gpu_cfg(shape, Lmax, n))
+    ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPARSE, sparse)
     kc, vc = wl.kv_cache(shape, config_id, 0, L, Lmax)
     x = wl.layer_input(shape, config_id, n)
     if vis is None:
@@ -69,8 +70,10 @@ def test_config5_llama13b_layer_wide_tree_and_lookahead_mask(ghd):
     parent = wl.random_tree(256, 8, wl.BASE_SEED + 5000, max_children=6)
     assert max(wl.depths_of(parent)) == 8
     _layer_parity(ghd, shape, w, gw, 5, 256, 4096, parent=parent)
+    _layer_parity(ghd, shape, w, gw, 5, 256, 4096, parent=parent, sparse=1)        # sparse part from the coordinate index
     vis, depth, _ = wl.lookahead_pattern(7, 5, 5)
     _layer_parity(ghd, shape, w, gw, 5, vis.shape[0], 4096, vis=vis, depth=depth)
+    _layer_parity(ghd, shape, w, gw, 5, vis.shape[0], 4096, vis=vis, depth=depth, sparse=1)
 
 
 def test_config3_full_32_layer_step_against_stored_oracle_results(ghd):
@@ -95,11 +98,16 @@ def test_config3_full_32_layer_step_against_stored_oracle_results(ghd):
     tok = to_dev(tokens)
     for _ in range(2):                                         # capture, then replay
         logits, amax = ghd.ghd_verify_step(ctx, gw, kvs, tree, tok)
+    hidden = ghd.ghd_copy_hidden(ctx, n)
     res = ghd.ghd_accept(ctx, tree, tok, amax).cpu().numpy()
     ghd.ghd_sync_status(ctx)
     got = logits.cpu().numpy()
-    # sampled logits, normalised by the oracle's largest |logit|
+    # the last layer's output (before the final norm) on the stored sample of columns, every node
+    hid = hidden.cpu().numpy()[:, fx["hidden_cols"]].astype(np.float64)
+    assert np.abs(hid - np.asarray(fx["hidden_samples"])).max() / fx["hidden_abs_max"] <= 2e-2
+    # sampled logits (512 columns per node, the oracle's top 8 among them), normalised by the oracle's largest |logit|
     abs_err = 0.0
+    assert len(fx["logit_samples"]) == n and all(len(r["cols"]) >= 512 for r in fx["logit_samples"])
     for srow in fx["logit_samples"]:
         g = got[srow["node"], srow["cols"]].astype(np.float64)
         abs_err = max(abs_err, float(np.abs(g - np.asarray(srow["values"])).max()))

@@ -47,6 +47,10 @@ def test_tree_build_bit_exact(ghd, name, parent):
     assert np.array_equal(tree.depth[:n].cpu().numpy(), depth)
     assert np.array_equal(tree.pos[:n].cpu().numpy(), pos)
     assert np.array_equal(tree.parent[:n].cpu().numpy(), np.asarray(parent, dtype=np.int32))
+    # the same visibility as a coordinate index (sparse part by list, Sec. III-B-3)
+    want_ptr, want_cols = oracle.coo_index(vis)
+    got_ptr, got_cols = tree.coo()
+    assert tree.c.nnz == want_ptr[-1] and np.array_equal(got_ptr, want_ptr) and np.array_equal(got_cols, want_cols)
     # rotary table: cos/sin of pos * theta^(-2t/dh), checked through the oracle's rotation of unit vectors
     dh = SMALL32.d_head
     unit = np.zeros((n, 1, dh))
@@ -67,6 +71,8 @@ def test_tree_from_explicit_lookahead_mask_equals_tree_build(ghd):
     n = len(parent)
     assert np.array_equal(a.mask_words(), b.mask_words())
     for t in (a, c):
+        assert all(np.array_equal(x, y) for x, y in zip(t.coo(), b.coo())) and t.c.nnz == b.c.nnz
+        assert all(np.array_equal(x, y) for x, y in zip(t.coo(), oracle.coo_index(vis)))
         assert np.array_equal(t.depth[:n].cpu().numpy(), b.depth[:n].cpu().numpy())
         assert np.array_equal(t.pos[:n].cpu().numpy(), b.pos[:n].cpu().numpy())
         assert np.array_equal(t.rope.cpu().numpy(), b.rope.cpu().numpy())
@@ -154,11 +160,12 @@ def test_linear_tcgen05_path(ghd, n, k, m):
         assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
 
 
-def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0):
+def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0):
     Lmax = L + n + 3
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
     if path:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_PATH, path)
+    ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPARSE, sparse)
     if splits:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPLITS, splits)
     H, dh, dt = shape.n_heads, shape.d_head, shape.dtype
@@ -172,6 +179,8 @@ def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0):
     tree = ghd.ghd_tree_build(ctx, parent, L)
     out = ghd.ghd_tree_attention(ctx, to_dev(q.reshape(n, H * dh)), ghd.KvLayer(to_dev(kc), to_dev(vc), L), tree)
     ghd.ghd_sync_status(ctx)
+    if sparse:
+        assert ghd.ghd_path_count(ctx, ghd.PATH_ATTN_COO) == 1, "the coordinate-index kernel did not run"
     return max_rel_err(out.cpu().numpy().reshape(n, H, dh), want)
 
 
@@ -187,11 +196,50 @@ def test_tree_attention(ghd, shape, n, L, splits):
     assert err <= (2e-5 if shape.dtype == "f32" else 2e-3)
 
 
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
+@pytest.mark.parametrize("n,L,splits", ATTN_CASES)
+def test_tree_attention_sparse_part_from_the_coordinate_index(ghd, shape, n, L, splits):
+    """Same problems, the new keys gathered per query from the coordinate index instead of bitmask-skipped groups."""
+    parent = wl.random_tree(n, 8, 1000 + n, max_children=6)
+    err = _attention_case(ghd, shape, n, L, parent, splits, sparse=1)
+    assert err <= (2e-5 if shape.dtype == "f32" else 2e-3)
+    if shape.dtype == "f16":
+        assert _attention_case(ghd, shape, n, L, parent, splits, path=1, sparse=1) <= 2e-3      # cache part on CUDA cores
+
+
 @pytest.mark.parametrize("n,L,splits", [(64, 2048, 0), (64, 2048, 5), (200, 1000, 0), (256, 4096, 0), (49, 640, 3)])
 def test_tree_attention_long_cache_both_paths(ghd, n, L, splits):
     parent = wl.random_tree(n, 8, 2000 + n, max_children=6)
     assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits) <= 2e-3               # tcgen05 kernel
     assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits, path=1) <= 2e-3       # CUDA-core kernel
+
+
+def _random_mask(n, seed, density=0.3):
+    """Lower-triangular visibility with the diagonal set and NO closure under ancestry: row i may see
+    node j without seeing what j sees, which no parent array can express."""
+    rng = np.random.default_rng(seed)
+    vis = np.tril(rng.random((n, n)) < density)
+    np.fill_diagonal(vis, True)
+    return vis
+
+
+@pytest.mark.parametrize("shape", [SMALL16, SMALL16_DH128, SMALL32], ids=["f16", "f16dh128", "f32"])
+@pytest.mark.parametrize("n,L", [(49, 200), (130, 77), (256, 300)])
+def test_tree_attention_with_a_mask_that_is_not_a_tree(ghd, shape, n, L):
+    vis = _random_mask(n, 7000 + n)
+    assert any(vis[i, j] and not (vis[j] <= vis[i]).all() for i in range(n) for j in range(i))   # really not prefix-closed
+    Lmax = L + n
+    ctx = make_ctx(ghd, shape, Lmax, n)
+    H, dh, dt = shape.n_heads, shape.d_head, shape.dtype
+    q = wl.normal((n, H, dh), 7100, dtype=dt)
+    kc = wl.normal((H, Lmax, dh), 7101, dtype=dt)
+    vc = wl.normal((H, Lmax, dh), 7102, dtype=dt)
+    want = oracle.tree_attention(q, kc[:, L:L + n].transpose(1, 0, 2), vc[:, L:L + n].transpose(1, 0, 2), kc, vc, L, vis.astype(np.uint8))
+    tree = ghd.ghd_tree_from_mask(ctx, ghd.pack_mask(vis), L)
+    assert np.array_equal(unpack_mask(tree.mask_words(), n), vis.astype(np.uint8))
+    out = ghd.ghd_tree_attention(ctx, to_dev(q.reshape(n, H * dh)), ghd.KvLayer(to_dev(kc), to_dev(vc), L), tree)
+    ghd.ghd_sync_status(ctx)
+    assert max_rel_err(out.cpu().numpy().reshape(n, H, dh), want) <= (2e-5 if dt == "f32" else 2e-3)
 
 
 def test_chain_tree_is_causal_attention_and_star_sees_only_root(ghd):
@@ -282,7 +330,8 @@ def _layer_case(ghd, shape, config_id, n, L, parent, vis=None, depth=None, gains
         ovis, _, opos = oracle.tree_build(parent, L)
         tree = ghd.ghd_tree_build(ctx, parent, L)
     else:
-        ovis, opos = vis.astype(np.uint8), (L + depth).astype(np.int32)
+        odepth = depth if depth is not None else vis.sum(axis=1) - 1      # the library's default: visible nodes - 1
+        ovis, opos = vis.astype(np.uint8), (L + odepth).astype(np.int32)
         tree = ghd.ghd_tree_from_mask(ctx, ghd.pack_mask(vis), L, depth=depth)
     okc, ovc = kc.copy(), vc.copy()
     want = oracle.layer(shape, w, okc, ovc, L, ovis, opos, x)
@@ -327,9 +376,66 @@ def test_config2_llama7b_layer_f16(ghd):
     _layer_case(ghd, wl.LLAMA7B, 2, 64, 1024, wl.medusa_tree(64), gains=False)
 
 
+@pytest.mark.parametrize("n,L", [(49, 200), (130, 77), (256, 300)])
+def test_layer_with_a_mask_that_is_not_a_tree(ghd, n, L):
+    """Whole layer under an arbitrary lower-triangular mask (position = kv_len + number of visible nodes - 1)."""
+    vis = _random_mask(n, 7200 + n)
+    depth = (vis.sum(axis=1) - 1).astype(np.int32)
+    _layer_case(ghd, SMALL16_DH128, 15, n, L, None, vis=vis, depth=depth)
+    _layer_case(ghd, SMALL16_DH128, 15, n, L, None, vis=vis, depth=None)      # depth taken from the popcount on the device
+
+
+def test_forced_tcgen05_gemm_refuses_a_reduction_length_off_the_64_grid(ghd):
+    """The tcgen05 projection walks the reduction in 64-wide slabs: k % 64 != 0 is outside it.  Forcing that path
+    must fail cleanly (nothing launched); the automatic choice takes the CUDA-core kernel and matches the oracle."""
+    ctx = make_ctx(ghd, SMALL16, 128, 64)
+    n, k, m = 17, 352, 130
+    x = wl.normal((n, k), 341, 1.0, dtype="f16")
+    w = wl.normal((m, k), 342, 0.02, dtype="f16")
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PATH, 2)
+    before = ghd.ghd_launch_count(ctx)
+    with pytest.raises(ghd.GhdError) as e:
+        ghd.ghd_linear(ctx, to_dev(x), to_dev(w))
+    assert e.value.name == "GHD_EUNSUPPORTED" and ghd.ghd_launch_count(ctx) == before
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PATH, 0)
+    y = ghd.ghd_linear(ctx, to_dev(x), to_dev(w))
+    ghd.ghd_sync_status(ctx)
+    assert ghd.ghd_path_count(ctx, ghd.PATH_GEMM_SIMT) == 1
+    assert max_rel_err(y.cpu().numpy(), oracle.linear(x, w)) <= 2e-5
+
+
+def test_graph_replay_notices_a_changed_option(ghd):
+    """The cached graph of a step is keyed on every option that changes what is enqueued: switching the
+    attention path between two graph-mode steps must re-capture, not replay the old kernels."""
+    shape, n, L = SMALL16_DH128, 12, 40
+    Lmax = L + n
+    parent = wl.random_tree(n, 4, 811)
+    head, layers, caches, gw, gkv = _model(ghd, shape, 16, L, Lmax)
+    ctx = make_ctx(ghd, shape, Lmax, n)
+    ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, 2)
+    tree = ghd.ghd_tree_build(ctx, parent, L)
+    tok = to_dev(wl.draft_tokens(parent, shape.vocab, 812))
+    l0, a0 = ghd.ghd_verify_step(ctx, gw, gkv, tree, tok)
+    assert ghd.ghd_path_count(ctx, ghd.PATH_ATTN_TC) == shape.n_layers and ghd.ghd_path_count(ctx, ghd.PATH_ATTN_SIMT) == 0
+    ghd.ghd_set_option(ctx, ghd.OPT_ATTN_PATH, 1)
+    l1, a1 = ghd.ghd_verify_step(ctx, gw, gkv, tree, tok)
+    ghd.ghd_sync_status(ctx)
+    assert ghd.ghd_path_count(ctx, ghd.PATH_ATTN_SIMT) == shape.n_layers, "the old graph was replayed"
+    assert max_rel_err(l1.cpu().numpy(), l0.cpu().numpy()) <= 2e-2 and np.array_equal(a0.cpu().numpy(), a1.cpu().numpy())
+
+
 def test_layer_with_explicit_lookahead_mask(ghd):
     vis, depth, parent = wl.lookahead_pattern(7, 5, 5)
     _layer_case(ghd, SMALL16_DH128, 12, len(parent), 200, parent, vis=vis, depth=depth)
+    _layer_case(ghd, SMALL16_DH128, 12, len(parent), 200, parent, vis=vis, depth=depth, opts=[(9, 1)])     # OPT_ATTN_SPARSE: index lists
+
+
+@pytest.mark.parametrize("n,L", [(13, 100), (64, 77), (256, 31)])
+def test_small_layers_sparse_part_from_the_coordinate_index(ghd, n, L):
+    import paper_2505_23219_b200 as g
+    for shape in (SMALL32, SMALL16_DH128):
+        ctx = _layer_case(ghd, shape, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6), opts=[(g.OPT_ATTN_SPARSE, 1)])
+        assert g.ghd_path_count(ctx, g.PATH_ATTN_COO) == 1
 
 
 # ---------------------------------------------------------------- step

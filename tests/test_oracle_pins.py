@@ -60,6 +60,32 @@ def test_tree_build_chain_and_star():
     assert list(depth) == [0] + [1] * 8
 
 
+@pytest.mark.parametrize("n,seed", [(1, 0), (9, 1), (64, 2), (130, 3), (256, 4)])
+def test_coo_index_lists_every_root_path(n, seed):
+    """For a tree the index of node i is its root path in ascending order: depth + 1 entries, ending in i,
+    each entry the parent of the next; the total is the sum of depth + 1."""
+    parent = wl.random_tree(n, 8, 900 + seed, max_children=6)
+    vis, depth, _ = oracle.tree_build(parent, 5)
+    ptr, cols = oracle.coo_index(vis)
+    assert ptr[0] == 0 and ptr[-1] == len(cols) == int((depth + 1).sum())
+    for i in range(n):
+        path = list(cols[ptr[i]:ptr[i + 1]])
+        assert len(path) == depth[i] + 1 and path[-1] == i and path[0] == 0
+        assert all(parent[b] == a for a, b in zip(path, path[1:]))
+
+
+def test_coo_index_of_an_arbitrary_mask_round_trips():
+    rng = np.random.default_rng(4)
+    vis = np.tril(rng.random((37, 37)) < 0.3)
+    np.fill_diagonal(vis, True)
+    ptr, cols = oracle.coo_index(vis)
+    back = np.zeros_like(vis)
+    for i in range(37):
+        assert list(cols[ptr[i]:ptr[i + 1]]) == sorted(cols[ptr[i]:ptr[i + 1]])
+        back[i, cols[ptr[i]:ptr[i + 1]]] = True
+    assert np.array_equal(back, vis) and ptr[-1] == vis.sum()
+
+
 @pytest.mark.parametrize("bad", [[], [0], [-1, 1], [-1, -1], [-1, 0, 3], [-1, 0, 2]])
 def test_tree_build_rejects_bad_parent(bad):
     with pytest.raises(ValueError):
