@@ -62,10 +62,10 @@ def algorithmic_bytes(shape, n, kv_len):
     return shape.n_layers * per_layer + shape.vocab * d * s + n * d * s + n * shape.vocab * 4
 
 
-# DRAM bytes per launch of the roofline kernel from the ncu capture summarised in
-# profiles/k_gemm_tc_gate_up_projection_llama7b.md; valid only for the kernel sources it was taken on.
-NCU_TRAFFIC = {"sources": ("gemm_tc.cu", "gemm_tc_dev.cuh", "tc_common.cuh"), "sha256_16": "32a19d9da7de0700",
-               "bytes_per_launch": 186.3e6}
+# DRAM bytes (read + written) per launch of the roofline kernel, from an ncu capture of exactly that launch;
+# valid only for the kernel sources it was taken on (hash below), else the line reports null.
+NCU_TRAFFIC = {"sources": ("gemm_tc.cu", "gemm_tc_dev.cuh", "tc_common.cuh"), "sha256_16": "8df6dc74085890c9",
+               "bytes_per_launch": 183.3e6}
 
 
 def ncu_traffic():
@@ -147,8 +147,12 @@ def time_oracle_sample(shape, n, kv_len, parent, tokens, sample_layers: int):
     oracle.accept(parent, tokens, amax)
     t_head = time.perf_counter() - t0
     est = t_layers * shape.n_layers / max(sample_layers, 1) + t_head
-    desc = (f"layers 0..{sample_layers - 1} of {shape.n_layers} timed ({t_layers:.2f} s) and scaled by "
-            f"{shape.n_layers}/{sample_layers}, plus final norm + lm_head + argmax + accept ({t_head:.2f} s)")
+    if sample_layers >= shape.n_layers:
+        desc = (f"one whole step: all {shape.n_layers} layers ({t_layers:.2f} s) + final norm + lm_head + argmax + accept "
+                f"({t_head:.2f} s), single run")
+    else:
+        desc = (f"layers 0..{sample_layers - 1} of {shape.n_layers} timed ({t_layers:.2f} s) and scaled by "
+                f"{shape.n_layers}/{sample_layers}, plus final norm + lm_head + argmax + accept ({t_head:.2f} s)")
     return est * 1e6, oracle.n_threads(), desc
 
 
@@ -281,26 +285,30 @@ def run_gpu(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1) / args.steps
 
-    # ---- dominant kernel alone: the gate/up projection of every layer, each a distinct cold matrix
+    # ---- dominant kernel alone, as the step launches it: the gate/up projection with the SwiGLU epilogue
+    # (half output), every layer's matrix in turn (each a distinct cold matrix), consecutive launches chained the
+    # way they are inside a step (the next kernel sets up while its predecessor drains)
     d, f = shape.d_model, shape.d_ffn
     xh = dev(wl.normal((n, d), 12345, 1.0, dtype="f16"))
-    yraw = torch.empty((n, 2 * f), dtype=torch.float32, device="cuda")
+    u_out = torch.empty((n, f), dtype=torch.float16, device="cuda")
     reps = 3
+    ghd.ghd_set_option(ctx, ghd.OPT_CHAIN_CALLS, 1)
     for lw in g_layers:
-        ghd.ghd_linear(ctx, xh, lw.t["w_gate_up"], yraw)
+        ghd.ghd_gate_up(ctx, xh, lw.t["w_gate_up"], u_out)
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     torch.cuda.nvtx.range_push("roofline")
     k0.record()
     for _ in range(reps):
         for lw in g_layers:
-            ghd.ghd_linear(ctx, xh, lw.t["w_gate_up"], yraw)
+            ghd.ghd_gate_up(ctx, xh, lw.t["w_gate_up"], u_out)
     k1.record()
     torch.cuda.nvtx.range_pop()
     torch.cuda.synchronize()
+    ghd.ghd_set_option(ctx, ghd.OPT_CHAIN_CALLS, 0)
     ghd.ghd_sync_status(ctx)
     kern_ms = k0.elapsed_time(k1) / (reps * len(g_layers))
-    kern_bytes = 2 * f * d * 2 + n * d * 2 + n * 2 * f * 4
+    kern_bytes = 2 * f * d * 2 + n * d * 2 + n * f * 2            # weights + activations in + SwiGLU output (half)
     peak, peak_kind = measured_peak()
 
     ms_per_step, e2e_ms, kern_ms = slowest_rank([ms_per_step, e2e_ms, kern_ms], dist, "cuda")
@@ -325,13 +333,13 @@ def run_gpu(args):
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": int(tokens.nbytes + parent_np.nbytes),
                     "d2h_bytes_per_step": int(res_d.numel() * 4)},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "k_gemm_tc (gate/up projection, [2*11008 x 4096] half, raw float output)",
+            "roofline": {"bound": "hbm", "kernel": "k_gemm_tc (gate/up projection [2*11008 x 4096] half with the SwiGLU epilogue, as the step launches it)",
                          "achieved": kern_bytes / (kern_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                          "frac": kern_bytes / (kern_ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
                          "us_per_launch": kern_ms * 1e3, "bytes_per_launch": kern_bytes, "traffic": ncu_traffic()},
         }
         if world == 1 and not args.no_cpu:
-            v, cores, desc = time_oracle_sample(shape, n, kv_len, parent, tokens, min(shape.n_layers, 8))
+            v, cores, desc = time_oracle_sample(shape, n, kv_len, parent, tokens, shape.n_layers)      # the whole step, once
             line["cpu_baseline"] = {"value": v, "unit": "us", "cores": cores, "kind": "oracle", "sample": desc}
         print(json.dumps(line), flush=True)
     if dist is not None:

@@ -60,6 +60,10 @@ typedef enum ghd_option {
                                  dependent launch overlap between consecutive kernels)        */
     GHD_OPT_GEMM_STAGES = 7,  /* pipeline stages of the tcgen05 GEMM (0 = automatic)          */
     GHD_OPT_GEMM_EPI = 8,     /* epilogue warp groups of the tcgen05 GEMM: 0 auto, 1, 2        */
+    GHD_OPT_CHAIN_CALLS = 10, /* 1 = the caller promises that whatever runs before a call on the stream does not
+                                 write anything the call reads ahead of its dependency wait (weights, cache
+                                 rows below kv_len): the first kernel of every call may then start while
+                                 its predecessor drains, like the kernels inside a call do (0 = it waits)  */
     GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
                                  Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
                                  nobody sees them (default); 1 = per-query list of visible nodes (the
@@ -243,11 +247,14 @@ ghd_status ghd_tree_fill_tokens(ghd_ctx *ctx, const int32_t *cand_dev, const ghd
 
 /* Building blocks of the layer, exposed for unit tests (same kernels the layer uses).
  * ghd_linear: y float [n][m] = x T[n][k] * w T[m][k]^T.
+ * ghd_gate_up: u T [n][d_ffn] = SiLU(h Wg^T) * (h Wu^T) for h T [n][d_model], w_gate_up T [2*d_ffn][d_model]
+ *   (gate rows, then up rows): the first half of the MLP block with its activation fused, as the layer runs it.
  * ghd_rmsnorm: out T [n][d_model] = RMSNorm(x float [n][d_model]) * g.
  * ghd_tree_attention: q T [n][n_heads*d_head] (rotated), caches already holding the
  *   n new rows at [kv_len, kv_len+n) -> out T [n][n_heads*d_head].
  * ghd_argmax: float [n][v] -> int32 [n]. */
 ghd_status ghd_linear(ghd_ctx *ctx, const void *x, const void *w, int32_t n, int32_t k, int32_t m, float *y);
+ghd_status ghd_gate_up(ghd_ctx *ctx, const void *h, const void *w_gate_up, int32_t n, void *u);
 ghd_status ghd_rmsnorm(ghd_ctx *ctx, const float *x, const void *g, int32_t n, void *out);
 ghd_status ghd_tree_attention(ghd_ctx *ctx, const void *q, const ghd_kv_layer *kv, const ghd_tree *tree, void *out);
 ghd_status ghd_argmax(ghd_ctx *ctx, const float *logits, int32_t n, int32_t v, int32_t *out);

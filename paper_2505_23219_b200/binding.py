@@ -17,18 +17,18 @@ __all__ = [
     "GhdError", "ModelCfg", "LayerWeights", "ModelWeights", "KvLayer", "Tree", "Ctx", "load_library",
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
-    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_copy_hidden", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
+    "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_copy_hidden", "ghd_gate_up", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
     "MedusaWeights", "GHD_MAX_TOPK",
     "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_ATTN_COO",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "OPT_CHAIN_CALLS", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
 GHD_MAX_TOPK = 16
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
-OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE = 7, 8, 9
+OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE, OPT_CHAIN_CALLS = 7, 8, 9, 10
 PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_ATTN_COO = 0, 1, 2, 3, 4
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
@@ -39,7 +39,7 @@ EXPORTS = [
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
     "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit",
-    "ghd_medusa_draft", "ghd_tree_fill_tokens", "ghd_copy_hidden",
+    "ghd_medusa_draft", "ghd_tree_fill_tokens", "ghd_copy_hidden", "ghd_gate_up",
 ]
 
 
@@ -111,6 +111,7 @@ def load_library(path: str | Path | None = None):
         "ghd_tree_fill_tokens": ([vp, vp, vp, vp, vp, i32, vp], C.c_int),
         "ghd_linear": ([vp, vp, vp, i32, i32, i32, vp], C.c_int),
         "ghd_rmsnorm": ([vp, vp, vp, i32, vp], C.c_int),
+        "ghd_gate_up": ([vp, vp, vp, i32, vp], C.c_int),
         "ghd_tree_attention": ([vp, vp, C.POINTER(_Kv), C.POINTER(_Tree), vp], C.c_int),
         "ghd_argmax": ([vp, vp, i32, i32, vp], C.c_int),
         "ghd_sync_status": ([vp], C.c_int),
@@ -364,6 +365,15 @@ def ghd_linear(ctx: Ctx, x, w, y=None):
         y = torch.empty((n, m), dtype=torch.float32, device=ctx.device)
     ctx._check(ctx.lib.ghd_linear(ctx.handle, x.data_ptr(), w.data_ptr(), n, k, m, y.data_ptr()))
     return y
+
+
+def ghd_gate_up(ctx: Ctx, h, w_gate_up, u=None):
+    """u [n][d_ffn] = SiLU(h Wg^T) * (h Wu^T) with the layer's own kernel (gate rows first in w_gate_up)."""
+    n = h.shape[0]
+    if u is None:
+        u = torch.empty((n, ctx.cfg.c.d_ffn), dtype=ctx.cfg.torch_dtype, device=ctx.device)
+    ctx._check(ctx.lib.ghd_gate_up(ctx.handle, h.data_ptr(), w_gate_up.data_ptr(), n, u.data_ptr()))
+    return u
 
 
 def ghd_rmsnorm(ctx: Ctx, x, g, out=None):

@@ -176,12 +176,12 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = c->opt_chain_calls = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
     c->pending.active = 0;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     c->attr_gemm = c->attr_attn = false;
     c->launches = 0;
     memset(c->path_count, 0, sizeof(c->path_count));
@@ -229,6 +229,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_GEMM_CTAS: c->opt_gemm_ctas = value; break;
         case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
         case GHD_OPT_GEMM_STAGES: if (value == 1 || value > 10) return GHD_EINVAL; c->opt_gemm_stages = value; break;
+        case GHD_OPT_CHAIN_CALLS: c->opt_chain_calls = value ? 1 : 0; break;
         case GHD_OPT_ATTN_SPARSE: if (value > 1) return GHD_EINVAL; c->opt_attn_sparse = value; break;
         case GHD_OPT_GEMM_EPI: if (value > 2) return GHD_EINVAL; c->opt_gemm_epi = value; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
@@ -295,7 +296,7 @@ ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer
     if (s != GHD_OK) return s;
     if (kv->len != tree->kv_len) return fail(c, GHD_EINVAL, "layer: kv.len differs from tree.kv_len");
     c->pending.active = 0;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     launch_load_x(c, x_in, tree->n);
     if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
     if (c->pending.active) launch_fold_pending(c, tree->n, nullptr, nullptr, x_out);
@@ -319,7 +320,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     }
     float* logits = logits_dev ? logits_dev : c->logits;
     c->pending.active = 0;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     if (c->opt_graph != 2) {
         if ((s = step_body(c, w, kv, tree, tokens_dev, logits, argmax_dev)) != GHD_OK) return s;
         return check_cuda(c, "verify_step");
@@ -330,7 +331,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope); push(tree->coo_ptr); push(tree->coo_col);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
-    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse})
+    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse, c->opt_chain_calls})
         key.push_back((uint64_t)(uint32_t)o);       // every option that changes what is enqueued
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
@@ -408,7 +409,7 @@ ghd_status ghd_medusa_draft(ghd_ctx* c, const ghd_medusa_weights* w, const ghd_a
         return fail(c, GHD_ENOSPACE, "medusa: workspace too small for the heads' activations");
     float* logits = logits_dev ? logits_dev : c->mlogits;
     c->pending.active = 0;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     launch_medusa_gather(c, result_dev, c->attnbuf);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = c->raw;
@@ -439,14 +440,28 @@ ghd_status ghd_linear(ghd_ctx* c, const void* x, const void* w, int32_t n, int32
     if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = y;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     ghd_status s = project(c, x, w, n, k, m, e, nullptr, nullptr);
     return s != GHD_OK ? s : check_cuda(c, "linear");
 }
 
+ghd_status ghd_gate_up(ghd_ctx* c, const void* h, const void* w_gate_up, int32_t n, void* u) {
+    if (!c || !h || !w_gate_up || !u || n < 1) return GHD_EINVAL;
+    if (n > c->cfg.max_nodes) return fail(c, GHD_ENOSPACE, "gate_up: n > max_nodes");
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    EpiArgs e{};
+    e.mode = EPI_SWIGLU; e.out_t = u;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
+    void* keep = c->ubuf;
+    c->ubuf = u;                     // the CUDA-core path writes its SwiGLU output through the context's buffer pointer
+    const ghd_status s = project(c, h, w_gate_up, n, c->cfg.d_model, 2 * c->cfg.d_ffn, e, nullptr, nullptr);
+    c->ubuf = keep;
+    return s != GHD_OK ? s : check_cuda(c, "gate_up");
+}
+
 ghd_status ghd_rmsnorm(ghd_ctx* c, const float* x, const void* g, int32_t n, void* out) {
     if (!c || !x || !g || !out || n < 1) return GHD_EINVAL;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     launch_rmsnorm(c, x, g, n, out);
     return check_cuda(c, "rmsnorm");
 }
@@ -456,14 +471,14 @@ ghd_status ghd_tree_attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv,
     if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
     ghd_status s = check_tree(c, tree);
     if (s != GHD_OK) return s;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     if ((s = attention(c, q, kv, tree, out)) != GHD_OK) return s;
     return check_cuda(c, "tree_attention");
 }
 
 ghd_status ghd_argmax(ghd_ctx* c, const float* logits, int32_t n, int32_t v, int32_t* out) {
     if (!c || !logits || !out || n < 1 || v < 1) return GHD_EINVAL;
-    c->entry_fresh = 1;
+    c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     launch_argmax(c, logits, n, v, out);
     return check_cuda(c, "argmax");
 }

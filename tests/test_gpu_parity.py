@@ -135,6 +135,22 @@ def test_linear_cuda_core_path(ghd, shape, n, k, m):
     assert max_rel_err(y.cpu().numpy(), oracle.linear(x, w)) <= 2e-6
 
 
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
+@pytest.mark.parametrize("n", [1, 19, 64, 130])
+def test_gate_up_with_fused_swiglu(ghd, shape, n):
+    """First half of the MLP block as the layer runs it: u = SiLU(h Wg^T) * (h Wu^T)."""
+    ctx = make_ctx(ghd, shape, 128, 256)
+    d, f, dt = shape.d_model, shape.d_ffn, shape.dtype
+    h = wl.normal((n, d), 351, 1.0, dtype=dt)
+    w = wl.normal((2 * f, d), 352, 0.05, dtype=dt)
+    u = ghd.ghd_gate_up(ctx, to_dev(h), to_dev(w))
+    ghd.ghd_sync_status(ctx)
+    gu = oracle.linear(h, w)
+    g, up = gu[:, :f], gu[:, f:]
+    want = g / (1.0 + np.exp(-g)) * up
+    assert max_rel_err(u.float().cpu().numpy(), want) <= (2e-6 if dt == "f32" else 2e-3)
+
+
 TC_SHAPES = [(1, 64, 128), (5, 256, 40), (16, 512, 256), (17, 320, 130), (64, 4096, 1024), (64, 11008, 512),
              (100, 1024, 1001), (128, 512, 384), (200, 2048, 256), (256, 1024, 640)]
 
