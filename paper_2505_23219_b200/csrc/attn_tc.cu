@@ -325,12 +325,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             mbar_wait(smem_u32(&sm->pv_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
             if (warp_live) {
                 tc_fence_after();
+                if constexpr (HD == 64) {                      // both 32-column reads in flight, one wait
+                    float v[64];
+                    const uint32_t a0 = tmem_base + TMEM_PV + b * DH + half * HD + lane_off;
+                    tc_ld32x2(a0, a0 + 32, v);
 #pragma unroll
-                for (int c0 = 0; c0 < HD; c0 += 32) {
-                    float v[32];
-                    tc_ld32(tmem_base + TMEM_PV + b * DH + half * HD + c0 + lane_off, v);
+                    for (int j = 0; j < 64; ++j) o[j] = fmaf(o[j], corr, v[j]);
+                } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                    for (int c0 = 0; c0 < HD; c0 += 32) {
+                        float v[32];
+                        tc_ld32(tmem_base + TMEM_PV + b * DH + half * HD + c0 + lane_off, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                    }
                 }
                 tc_fence_before();
             }
@@ -458,11 +466,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             if (warp_live) {
                 tc_fence_after();
 #pragma unroll
-                for (int c0 = 0; c0 < DH; c0 += 32) {
-                    float v[32];
-                    tc_ld32(tmem_base + TMEM_PV + b * DH + c0 + lane_off, v);
+                for (int c0 = 0; c0 < DH; c0 += 64) {          // two 32-column reads in flight per wait
+                    float v[64];
+                    const uint32_t a0 = tmem_base + TMEM_PV + b * DH + c0 + lane_off;
+                    tc_ld32x2(a0, a0 + 32, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
+                    for (int j = 0; j < 64; ++j) o[c0 + j] = fmaf(o[c0 + j], corr, v[j]);
                 }
                 tc_fence_before();
             }
@@ -490,15 +499,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             }
             tc_fence_after();
             float s[BN];
-            {
-                float t[32];
-                tc_ld32(tmem_base + TMEM_S + b * BN + lane_off, t);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) s[j] = t[j];
-                tc_ld32(tmem_base + TMEM_S + b * BN + 32 + lane_off, t);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) s[32 + j] = t[j];
-            }
+            tc_ld32x2(tmem_base + TMEM_S + b * BN + lane_off, tmem_base + TMEM_S + b * BN + 32 + lane_off, s);
             tc_fence_before();
             mbar_arrive(smem_u32(&sm->s_empty[b]));
             // hidden keys become -inf once; exp2(-inf) = 0 then needs no further selects
