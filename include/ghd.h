@@ -64,6 +64,10 @@ typedef enum ghd_option {
                                  write anything the call reads ahead of its dependency wait (weights, cache
                                  rows below kv_len): the first kernel of every call may then start while
                                  its predecessor drains, like the kernels inside a call do (0 = it waits)  */
+    GHD_OPT_FUSED_NORM = 11,  /* tcgen05 path: 1 = the RMSNorms live in the projections' epilogues (the projection into
+                                 the residual stream leaves gain-weighted rows and per-tile sums of squares, its
+                                 consumer multiplies by 1 / rms); 0 = separate reduction + norm kernels (default:
+                                 faster as measured, the split tiles of the narrow projections finish in parallel)  */
     GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
                                  Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
                                  nobody sees them (default); 1 = per-query list of visible nodes (the
@@ -118,13 +122,26 @@ typedef struct ghd_kv_layer {
  *   the visible new nodes of query i are coo_col[coo_ptr[i] .. coo_ptr[i + 1]), ascending; nnz = coo_ptr[n].
  * GHD_OPT_ATTN_SPARSE = 1 needs it. */
 typedef struct ghd_tree {
-    int32_t n, kv_len, n_words, has_parent;
+    int32_t n, kv_len, n_words, has_parent;       /* kv_len = GHD_KV_LEN_DEVICE: taken from the context's device word */
     uint64_t *mask;
     int32_t *parent, *depth, *pos;
     float *rope;
     int32_t *coo_ptr, *coo_col;
     int32_t nnz;
 } ghd_tree;
+
+/* The cache length kept on the device (paper Sec. II-A: every step extends the cache by the tokens it
+ * produced; Sec. II-C: by the accepted ones only).  A context owns one int32 device word.  Wherever a call
+ * takes a cache length (ghd_tree_build, ghd_tree_from_mask, ghd_kv_layer.len, ghd_kv_commit) the value
+ * GHD_KV_LEN_DEVICE means "read the word on the device when the kernel runs": positions, the rows a step
+ * appends and the keys the attention walks then follow the word, and ghd_kv_commit advances it by
+ * n_matched + 1, so that a loop of draft / verify / accept / commit steps needs no host read between
+ * steps (and, with GHD_OPT_GRAPH = 2, replays one graph for every step).  Every kernel clamps the word to
+ * [0, max_kv_len - n]; the tree kernels record a word outside that range in the status word
+ * (ghd_sync_status -> GHD_ENOSPACE).  In this mode the attention kernels may fetch cache rows past
+ * kv_len + n (their weights are exactly zero): every row of the cache buffers must hold finite numbers,
+ * e.g. buffers that were zero-filled when they were allocated. */
+#define GHD_KV_LEN_DEVICE (-1)
 
 /* dev struct written by ghd_accept.  nodes[0..n_matched] is the accepted root
  * path (nodes[0] = 0); tokens[j] = argmax at nodes[j]; n_emitted = n_matched + 1
@@ -211,10 +228,18 @@ ghd_status ghd_accept(ghd_ctx *ctx, const ghd_tree *tree, const int32_t *tokens_
  * cache of the accepted sequence; later rows keep stale tree rows.  `result_dev` is the struct
  * ghd_accept filled (read on the device: no host round trip).  kv[l].len is a host field and is
  * NOT changed: the caller raises it to kv_len + n_matched + 1 once it has read n_matched.
+ * With kv_len = GHD_KV_LEN_DEVICE the rows move relative to the context's device word, which is then
+ * advanced to word + n_matched + 1 (clamped to max_kv_len - 1) by a kernel enqueued behind the moves.
  * Enqueued on the context's stream.  GHD_EINVAL on null pointers, GHD_ENOSPACE when
  * kv_len + max_nodes > max_kv_len could be exceeded (kv_len < 0 or kv_len + 1 > max_kv_len). */
 ghd_status ghd_kv_commit(ghd_ctx *ctx, const ghd_kv_layer *kv, int32_t n_layers, int32_t kv_len,
                          const ghd_accept_result *result_dev);
+
+/* The device word with the cache length (see GHD_KV_LEN_DEVICE). */
+/* Sets the word (enqueued on the context's stream).  GHD_ENOSPACE: no workspace, or kv_len outside [0, max_kv_len). */
+ghd_status ghd_kv_len_set(ghd_ctx *ctx, int32_t kv_len);
+/* Waits for the context's stream and copies the word to *kv_len_host. */
+ghd_status ghd_kv_len_get(ghd_ctx *ctx, int32_t *kv_len_host);
 
 /* Self-drafting with extra heads (paper Sec. II-C: Medusa-style heads attached after the last layer each
  * draft the token of one later position; the paper's default drafter).  The paper does not

@@ -18,17 +18,18 @@ __all__ = [
     "ghd_create", "ghd_destroy", "ghd_set_option", "ghd_tree_build", "ghd_tree_from_mask", "ghd_verify_layer",
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
     "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_copy_hidden", "ghd_gate_up", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
-    "MedusaWeights", "GHD_MAX_TOPK",
+    "ghd_kv_len_set", "ghd_kv_len_get", "KV_LEN_DEVICE", "MedusaWeights", "GHD_MAX_TOPK",
     "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_ATTN_COO",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
-    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "OPT_CHAIN_CALLS", "EXPORTS",
+    "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "OPT_CHAIN_CALLS", "OPT_FUSED_NORM", "EXPORTS",
 ]
 
 GHD_F32, GHD_F16 = 0, 1
 GHD_MAX_NODES = 256
 GHD_MAX_TOPK = 16
+KV_LEN_DEVICE = -1      # "take the cache length from the context's device word"
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
-OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE, OPT_CHAIN_CALLS = 7, 8, 9, 10
+OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE, OPT_CHAIN_CALLS, OPT_FUSED_NORM = 7, 8, 9, 10, 11
 PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_ATTN_COO = 0, 1, 2, 3, 4
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
@@ -38,7 +39,7 @@ EXPORTS = [
     "ghd_create", "ghd_destroy", "ghd_workspace_bytes", "ghd_set_workspace", "ghd_set_option", "ghd_tree_build",
     "ghd_tree_from_mask", "ghd_verify_layer", "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm",
     "ghd_tree_attention", "ghd_argmax", "ghd_sync_status", "ghd_status_str", "ghd_last_error", "ghd_launch_count",
-    "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit",
+    "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_kv_len_set", "ghd_kv_len_get",
     "ghd_medusa_draft", "ghd_tree_fill_tokens", "ghd_copy_hidden", "ghd_gate_up",
 ]
 
@@ -107,6 +108,8 @@ def load_library(path: str | Path | None = None):
         "ghd_accept": ([vp, C.POINTER(_Tree), vp, vp, vp], C.c_int),
         "ghd_copy_hidden": ([vp, i32, vp], C.c_int),
         "ghd_kv_commit": ([vp, C.POINTER(_Kv), i32, i32, vp], C.c_int),
+        "ghd_kv_len_set": ([vp, i32], C.c_int),
+        "ghd_kv_len_get": ([vp, C.POINTER(i32)], C.c_int),
         "ghd_medusa_draft": ([vp, C.POINTER(_MedusaW), vp, vp, vp, vp], C.c_int),
         "ghd_tree_fill_tokens": ([vp, vp, vp, vp, vp, i32, vp], C.c_int),
         "ghd_linear": ([vp, vp, vp, i32, i32, i32, vp], C.c_int),
@@ -334,6 +337,18 @@ def ghd_kv_commit(ctx: Ctx, kvs, kv_len: int, result):
     kv_len .. kv_len + n_matched in every layer of `kvs`.  The layers' `len` fields are left alone."""
     arr = (_Kv * len(kvs))(*[kv.c for kv in kvs])
     ctx._check(ctx.lib.ghd_kv_commit(ctx.handle, arr, len(kvs), kv_len, result.data_ptr()))
+
+
+def ghd_kv_len_set(ctx: Ctx, kv_len: int):
+    """Writes the context's device word with the cache length (read by calls given KV_LEN_DEVICE)."""
+    ctx._check(ctx.lib.ghd_kv_len_set(ctx.handle, int(kv_len)))
+
+
+def ghd_kv_len_get(ctx: Ctx) -> int:
+    """Waits for the stream and reads the device word back."""
+    out = C.c_int32(0)
+    ctx._check(ctx.lib.ghd_kv_len_get(ctx.handle, C.byref(out)))
+    return int(out.value)
 
 
 def ghd_medusa_draft(ctx: Ctx, w: MedusaWeights, result, topk, want_logits: bool = False):

@@ -33,8 +33,13 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(QB * 32)
 k_attn_simt(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
             const uint64_t* __restrict__ mask, int n_words, int n, int n_new, int heads, int kv_len, int max_kv,
-            int chunk, float* __restrict__ part_o, float* __restrict__ part_ml, int max_nodes) {
+            int chunk, float* __restrict__ part_o, float* __restrict__ part_ml, int max_nodes, const int* __restrict__ kv_len_dev) {
     constexpr int R = DH / 32;
+    if (kv_len_dev) {          // the length lives on the device: deal the keys to the splits here
+        kv_len = resolve_kv_len(kv_len, kv_len_dev, max_kv, n);
+        chunk = (kv_len + n_new + (int)gridDim.z - 1) / (int)gridDim.z;
+        chunk = ((chunk + TK - 1) / TK) * TK;
+    }
     __shared__ float sq[QB][DH];
     __shared__ float sk[TK][DH + 1];
     __shared__ float sv[TK][DH + 1];
@@ -135,10 +140,11 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(COO_WARPS * 32)
 k_attn_coo(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc, const int32_t* __restrict__ coo_ptr,
            const int32_t* __restrict__ coo_col, int n, int heads, int kv_len, int max_kv,
-           float* __restrict__ part_o, float* __restrict__ part_ml) {
+           float* __restrict__ part_o, float* __restrict__ part_ml, const int* __restrict__ kv_len_dev) {
     constexpr int R = DH / 32;
     pdl_wait();
     pdl_trigger();
+    kv_len = resolve_kv_len(kv_len, kv_len_dev, max_kv, n);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i = blockIdx.x * COO_WARPS + warp, h = blockIdx.y;
     if (i >= n) return;
@@ -264,7 +270,7 @@ int attn_auto_splits(const ghd_ctx* c, int n, int kv_total) {
 void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo) {
     const ghd_model_cfg& m = c->cfg;
     const int n_new = coo ? 0 : t->n;
-    const int kt = t->kv_len + n_new;
+    const int kt = kv_len_host_of(c, t) + n_new;
     int splits = c->opt_attn_splits > 0 ? c->opt_attn_splits : attn_auto_splits(c, t->n, kt);
     if (splits > c->max_splits - (coo ? 1 : 0)) splits = c->max_splits - (coo ? 1 : 0);
     int chunk = (kt + splits - 1) / splits;
@@ -273,7 +279,7 @@ void launch_attn_simt(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const g
 #define GHD_ATTN(T, DH)                                                                                          \
     k_attn_simt<T, DH><<<grid, QB * 32, 0, c->cur>>>((const T*)q, (const T*)kv->k, (const T*)kv->v, t->mask,  \
                                                         t->n_words, t->n, n_new, m.n_heads, t->kv_len, m.max_kv_len, \
-                                                        chunk, c->att_o, c->att_ml, m.max_nodes)
+                                                        chunk, c->att_o, c->att_ml, m.max_nodes, kv_len_dev_of(c, t))
     if (m.dtype == GHD_F32) { if (m.d_head == 64) GHD_ATTN(float, 64); else GHD_ATTN(float, 128); }
     else { if (m.d_head == 64) GHD_ATTN(__half, 64); else GHD_ATTN(__half, 128); }
 #undef GHD_ATTN
@@ -295,7 +301,8 @@ void launch_attn_coo(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const gh
 #define GHD_COO(T, DH)                                                                                              \
     launch_k(c, true, k_attn_coo<T, DH>, grid, dim3(COO_WARPS * 32), 0, (const T*)q, (const T*)kv->k, (const T*)kv->v,   \
              (const int32_t*)t->coo_ptr, (const int32_t*)t->coo_col, t->n, m.n_heads, t->kv_len, m.max_kv_len,      \
-             c->att_o + (size_t)slot * m.max_nodes * m.d_model, c->att_ml + (size_t)slot * m.max_nodes * m.n_heads * 2)
+             c->att_o + (size_t)slot * m.max_nodes * m.d_model, c->att_ml + (size_t)slot * m.max_nodes * m.n_heads * 2, \
+             kv_len_dev_of(c, t))
     if (m.dtype == GHD_F32) { if (m.d_head == 64) GHD_COO(float, 64); else GHD_COO(float, 128); }
     else { if (m.d_head == 64) GHD_COO(__half, 64); else GHD_COO(__half, 128); }
 #undef GHD_COO
@@ -412,7 +419,7 @@ extern "C" ghd_status ghd_tree_attention_static(void* cuda_stream, int32_t dtype
 #define GHD_ATTN_ST(T, DH)                                                                                  \
     k_attn_simt<T, DH><<<grid, QB * 32, 0, stream>>>((const T*)q, (const T*)k_cache, (const T*)v_cache,      \
                                                      mask_dev, n_words, n, n, n_heads, kv_len, max_kv_len,   \
-                                                     chunk, part_o, part_ml, ST_MAX_NODES)
+                                                     chunk, part_o, part_ml, ST_MAX_NODES, (const int*)nullptr)
     if (dtype == GHD_F32) { if (d_head == 64) GHD_ATTN_ST(float, 64); else GHD_ATTN_ST(float, 128); }
     else { if (d_head == 64) GHD_ATTN_ST(__half, 64); else GHD_ATTN_ST(__half, 128); }
 #undef GHD_ATTN_ST

@@ -44,6 +44,8 @@ constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 
 struct AttnParams {
     int n, heads, kv_len, max_nodes, splits, n_words;
+    const int* kv_len_dev;     // non-null: the cache length comes from this device word
+    int max_kv_len;
     int cache_only;            // 1: the new rows are somebody else's (the coordinate-index kernel): no node groups here
     const uint64_t* mask;
     float* part_o;
@@ -142,7 +144,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // row of the CTA can see.  Which groups are visible is known only after the mask rows have
     // arrived; every role waits for that (mask_ready) when it reaches the first node group, so
     // the mask's load latency hides behind the cache tiles.
-    const int n_cache = (p.kv_len + BN - 1) / BN;
+    // (a length kept on the device was written at least two kernels ago: it may be read ahead of the dependency wait)
+    const int kv_len = resolve_kv_len(p.kv_len, p.kv_len_dev, p.max_kv_len, p.n);
+    const int n_cache = (kv_len + BN - 1) / BN;
     const int c_beg = n_cache * split / p.splits, c_end = n_cache * (split + 1) / p.splits;
     uint32_t cand = 0;
 #pragma unroll
@@ -160,7 +164,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
             for (int w = 0; w < MAX_UNITS_WORDS; ++w)
                 if (((cand >> w) & 1u) && sm->word_or[w] != 0ull) {
-                    if (!body(i, p.kv_len + 64 * w, w)) return i;
+                    if (!body(i, kv_len + 64 * w, w)) return i;
                     ++i;
                 }
         }
@@ -185,7 +189,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             // cache tiles wholly below kv_len are not written by the preceding kernel: request the
             // first ring-full of them before waiting for that kernel to finish
             int pre = 0;
-            for (int c = c_beg; c < c_end && pre < KV_STAGES && (c + 1) * BN <= p.kv_len; ++c, ++pre) load_kv(pre, c * BN);
+            for (int c = c_beg; c < c_end && pre < KV_STAGES && (c + 1) * BN <= kv_len; ++c, ++pre) load_kv(pre, c * BN);
             pdl_wait();
             uint32_t stage = 0, phase = 0;
             int issued = 0;
@@ -350,7 +354,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             // visibility of this thread's 32 keys
             uint32_t bits = 0u;
             if (w < 0) {
-                const int valid = p.kv_len - key0 - half * HC;
+                const int valid = kv_len - key0 - half * HC;
                 if (live) bits = valid >= HC ? 0xffffffffu : (valid > 0 ? ((1u << valid) - 1u) : 0u);
             } else {
 #pragma unroll
@@ -483,7 +487,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             // visibility of the 64 keys of this unit for this row
             unsigned long long vis = 0ull;
             if (w < 0) {
-                const int valid = p.kv_len - key0;
+                const int valid = kv_len - key0;
                 if (live) vis = valid >= 64 ? ~0ull : ((1ull << valid) - 1ull);
             } else {
 #pragma unroll
@@ -576,7 +580,9 @@ bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t) {
 ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo) {
     const ghd_model_cfg& m = c->cfg;
     const int n = t->n, H = m.n_heads, dh = m.d_head, d = m.d_model;
-    const int kt = t->kv_len + n;
+    // rows the K/V maps cover: past them a load returns zeros.  With the length on the device the maps cover the
+    // whole cache and rows past kv_len + n (weight exactly zero) must hold finite numbers.
+    const int kt = t->kv_len < 0 ? m.max_kv_len : t->kv_len + n;
     if (((uintptr_t)q & 15) || ((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: operands must be 16-byte aligned");
         return GHD_EINVAL;
@@ -590,7 +596,7 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         return GHD_ECUDA;
     }
     const int mtiles = (n + QM - 1) / QM;
-    const int units = (t->kv_len + BN - 1) / BN + (coo ? 0 : t->n_words);
+    const int units = (kv_len_host_of(c, t) + BN - 1) / BN + (coo ? 0 : t->n_words);
     int splits = c->opt_attn_splits;
     if (splits <= 0) {
         splits = c->sm_count / (H * mtiles);
@@ -601,7 +607,7 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
     if (splits < 1) splits = 1;
     AttnParams p{};
     p.cache_only = coo ? 1 : 0;
-    p.n = n; p.heads = H; p.kv_len = t->kv_len; p.max_nodes = m.max_nodes; p.splits = splits; p.n_words = t->n_words;
+    p.n = n; p.heads = H; p.kv_len = t->kv_len; p.kv_len_dev = kv_len_dev_of(c, t); p.max_kv_len = m.max_kv_len; p.max_nodes = m.max_nodes; p.splits = splits; p.n_words = t->n_words;
     p.mask = t->mask; p.part_o = c->att_o; p.part_ml = c->att_ml; p.status = c->status;
     p.scale = 1.0f / sqrtf((float)dh);
     dim3 grid(splits, H, mtiles);

@@ -197,11 +197,48 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         auto epi_all = [] { if (TWO) all_epi_bar(); else grp_bar(0); };
         auto fused = [&](int tile_, int c0_, float (&v_)[32]) { epilogue_chunk<GROUPS>(p, sm, grp, tile_, row, c0_, v_); };
         const int et = threadIdx.x - 64;                       // 0..255 among epilogue threads
+        const size_t slot_elems = (size_t)buf_cols * TILE_M;   // columns padded to whole 32-wide chunks
+        // Epilogue of a complete tile.  split = false: the accumulator holds the whole sum.  split = true: this CTA
+        // (the tile's first contributor) has its share in tensor memory and adds the other contributors' partial
+        // tiles from the workspace in CTA order (fixed order -> reproducible); each one's 32 loads go out together.
+        auto finish_tile = [&](int tile_, uint32_t t_addr_, bool split, int c_first_, int c_last_) {
+            for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += GROUPS * EPI_CHUNK) {
+                float v[32];
+                tc_ld32(t_addr_ + c0, v);                  // may run past nb, never past the buffer
+                if (split) {
+                    for (int c = c_first_ + 1; c <= c_last_; ++c) {      // later contributors always use their slot 0
+                        const float* src = p.part + (size_t)c * 2 * slot_elems + (size_t)c0 * TILE_M + row;
+                        float t[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * TILE_M);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += t[j];
+                    }
+                }
+                fused(tile_, c0, v);
+            }
+        };
         pdl_wait();                                            // outputs, residual and partial buffers belong to earlier kernels until now
+        if (p.epi.ssq_in) {
+            // 1 / rms of every input row from the per-tile sums of squares its producer left (fixed order)
+            for (int i = et; i < p.nb; i += TWO ? 256 : 128) {
+                float s = 0.f;
+                if (i < p.n)
+                    for (int t0 = 0; t0 < p.epi.ssq_in_tiles; t0 += 8) {
+                        float part[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            part[q] = (t0 + q < p.epi.ssq_in_tiles) ? __ldcg(p.epi.ssq_in + (size_t)(t0 + q) * SSQ_PITCH + i) : 0.f;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) s += part[q];
+                    }
+                sm->colscale[i] = rsqrtf(s / (float)p.k + p.epi.rms_eps);
+            }
+            epi_all();
+        }
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
         long long it = it_beg;
-        const size_t slot_elems = (size_t)buf_cols * TILE_M;   // columns padded to whole 32-wide chunks
         int tile = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)tile * p.kiters);
         for (; it < it_end && ok; ++tile, k0 = 0) {
             const long long left = it_end - it;
@@ -213,94 +250,54 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
-            if (whole) {
-                for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += GROUPS * EPI_CHUNK) {
-                    float v[32];
-                    tc_ld32(t_addr + c0, v);                   // may run past nb, never past the buffer
-                    if (c0 < p.n) fused(tile, c0, v);
+            // A tile some CTAs share is finished by its FIRST contributor: for that CTA the tile is the last unit of
+            // its range, so it gets here last in time, while every other contributor handles its share as the first
+            // unit of its range (or as its only one), stores it and counts itself in without ever waiting.  The
+            // finisher keeps its own share in tensor memory and waits (bounded) for the others; they run at the same
+            // time on other SMs and depend on nobody, so the wait is short: the store and count of a contributor
+            // that ended together with the finisher.
+            const int c_first = p.tile_first[tile], c_last = c_first + p.tile_count[tile] - 1;
+            bool finish = whole;
+            if (!whole && p.epi.mode != EPI_DEFER) {
+                if (et == 0) {
+                    int fl = 0;
+                    if (cta == c_first) {
+                        fl = 1;
+                        uint32_t spin = 0;
+                        while (ld_acquire_gpu(p.counters + tile) != c_last - c_first) {
+                            if (++spin >= SPIN_LIMIT) { *abort_flag = 1; atomicCAS(p.status, DEV_OK, DEV_TIMEOUT_GRID); break; }
+                            __nanosleep(spin > 64 ? 64 : 20);
+                        }
+                    }
+                    sm->last_flag = fl;
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+                epi_all();
+                finish = sm->last_flag != 0;
+                epi_all();
+            }
+            if (finish) {
+                finish_tile(tile, t_addr, !whole, c_first, c_last);
+                if (!whole && et == 0) p.counters[tile] = 0;   // ready for the next launch
             } else {
                 // partial tile: slot 0 when this is the CTA's first unit (it starts mid-tile or is
                 // its only unit of this tile), slot 1 when it is the head part of the CTA's last tile
                 const int slot = (it == it_beg) ? 0 : 1;
                 float* mine = p.part + ((size_t)cta * 2 + slot) * slot_elems;
-                const int c_first = p.tile_first[tile], c_last = c_first + p.tile_count[tile] - 1;
-                bool finish = false;       // this CTA completes the tile
-                bool dumped = false;
-                if (p.epi.mode != EPI_DEFER) {
-                    // The tile is finished by its FIRST contributor: for that CTA the tile is the last unit of its
-                    // range, so it gets here last in time, while every other contributor handles its share as the
-                    // first unit of its range (or as its only one), stores it and counts itself in without ever
-                    // waiting.  The finisher keeps its own share in tensor memory and waits (bounded) for the
-                    // others; they run at the same time on other SMs and depend on nobody, so the wait is short:
-                    // the store and count of a contributor that ended together with the finisher.
-                    if (et == 0) {
-                        int fl = 0;
-                        if (cta == c_first) {
-                            fl = 1;
-                            uint32_t spin = 0;
-                            while (ld_acquire_gpu(p.counters + tile) != c_last - c_first) {
-                                if (++spin >= SPIN_LIMIT) { *abort_flag = 1; atomicCAS(p.status, DEV_OK, DEV_TIMEOUT_GRID); break; }
-                                __nanosleep(spin > 64 ? 64 : 20);
-                            }
-                        }
-                        sm->last_flag = fl;
-                    }
-                    epi_all();
-                    finish = sm->last_flag != 0;
-                    epi_all();
+                for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += GROUPS * EPI_CHUNK) {
+                    float v[32];
+                    tc_ld32(t_addr + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
                 }
-                if (!finish) {
-                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb; c0 += GROUPS * EPI_CHUNK) {
-                        float v[32];
-                        tc_ld32(t_addr + c0, v);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
-                    }
-                    dumped = true;
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
-                    if (p.epi.mode != EPI_DEFER) {
-                        // count this arrival: the barrier orders every thread's stores before thread 0's
-                        // release, and the release is cumulative over them
-                        epi_all();
-                        if (et == 0) atom_add_acq_rel_gpu(p.counters + tile, 1);
-                    }
-                }
-                if (finish) {
-                    for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += GROUPS * EPI_CHUNK) {
-                        float v[32], own[32];
-                        if (!dumped) tc_ld32(t_addr + c0, own);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                        // contributors in CTA order (fixed order -> reproducible); each one's 32 loads go out together
-                        for (int c = c_first; c <= c_last; ++c) {
-                            if (c == cta && !dumped) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) v[j] += own[j];
-                                continue;
-                            }
-                            const int cslot = (c == c_first) ? p.tile_slot[tile] : 0;
-                            const float* src = p.part + ((size_t)c * 2 + cslot) * slot_elems + (size_t)c0 * TILE_M + row;
-                            float t[32];
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * TILE_M);
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] += t[j];
-                        }
-                        fused(tile, c0, v);
-                    }
-                    if (!dumped) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
-                    }
-                    if (et == 0) p.counters[tile] = 0;         // ready for the next launch
-                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+            if (!finish && p.epi.mode != EPI_DEFER) {
+                // count this arrival: the barrier orders every thread's stores before thread 0's
+                // release, and the release is cumulative over them
+                epi_all();
+                if (et == 0) atom_add_acq_rel_gpu(p.counters + tile, 1);
             }
             if (++buf == 2) { buf = 0; buf_phase ^= 1; }
             it += (k1 - k0);
@@ -334,6 +331,7 @@ bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
     if (n_tiles < 1 || n_tiles > MAX_TILES) return false;
     if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
     if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
+    if (epi_mode == EPI_RESID_NORM && (m % TILE_M || m / TILE_M > SSQ_MAX_TILES)) return false;
     if (epi_mode == EPI_DEFER) {
         int ctas = c->opt_gemm_ctas > 0 && c->opt_gemm_ctas < c->sm_count ? c->opt_gemm_ctas : c->sm_count;
         const int ks = (((n + 15) / 16) * 16 <= 128) ? 2 : 1;

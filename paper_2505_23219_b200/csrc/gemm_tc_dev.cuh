@@ -45,7 +45,31 @@ struct Smem {
     int abort_flag;
     int last_flag;
     float stage_x[EPI_CHUNK][TILE_M + 1];   // epilogue exchange buffer (rotary pairs, gate/up pairs)
+    float colscale[GHD_MAX_NODES];          // 1 / rms of every input row (projections that read un-normalised rows)
+    float ssq_part[2][4][32];               // per epilogue group and warp: sums of squares of 32 rows x 32 nodes
 };
+
+// s[j] (j < 32) summed over the 32 lanes of the warp; lane L returns the total of column L.
+// Each step halves the columns a lane is responsible for: 16 + 8 + 4 + 2 + 1 shuffles.
+template <int N>
+__device__ __forceinline__ void warp_transpose_sum_step(float (&s)[32], int lane) {
+    constexpr int H = N / 2;
+    const bool up = (lane & H) != 0;
+#pragma unroll
+    for (int i = 0; i < H; ++i) {
+        const float send = up ? s[i] : s[i + H];
+        const float keep = up ? s[i + H] : s[i];
+        s[i] = keep + __shfl_xor_sync(0xffffffffu, send, H);
+    }
+}
+__device__ __forceinline__ float warp_transpose_sum(float (&s)[32], int lane) {
+    warp_transpose_sum_step<32>(s, lane);
+    warp_transpose_sum_step<16>(s, lane);
+    warp_transpose_sum_step<8>(s, lane);
+    warp_transpose_sum_step<4>(s, lane);
+    warp_transpose_sum_step<2>(s, lane);
+    return s[0];
+}
 
 // ---------------------------------------------------------------- fused epilogue
 // Thread `row` (0..127) of the tile holds the final sums v[j] of its output feature for nodes
@@ -63,6 +87,40 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
     constexpr int PASSES = GROUPS;
     const EpiArgs& e = p.epi;
     float (*xb)[TILE_M + 1] = sm->stage_x + grp * XR;
+    if (e.ssq_in) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] *= sm->colscale[c0 + j];
+    }
+    if (e.mode == EPI_RESID_NORM) {
+        // residual add, the gain-weighted copy for the next projection, and this tile's share of every
+        // node's sum of squares (the consumer turns the sums into 1 / rms); m is a multiple of 128
+        const int f = tile * TILE_M + row, lane = row & 31, quad = row >> 5;
+        float* xr = e.out_f32 + (size_t)c0 * p.m + f;
+        __half* xg = (__half*)e.xg_out + (size_t)c0 * p.m + f;
+        const unsigned m = (unsigned)p.m;
+        {
+            float old[32];      // all loads first: a load after a store through another pointer would wait for it
+#pragma unroll
+            for (int j = 0; j < 32; ++j) old[j] = (c0 + j < p.n) ? __ldcg(xr + j * m) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (c0 + j < p.n) ? v[j] + old[j] : 0.f;
+        }
+        const float g = __half2float(__ldg((const __half*)e.gain + f));
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (c0 + j < p.n) {
+                xr[j * m] = v[j];
+                xg[j * m] = __float2half_rn(v[j] * g);
+                v[j] *= v[j];
+            }
+        sm->ssq_part[grp][quad][lane] = warp_transpose_sum(v, lane);
+        grp_bar(grp);
+        if (quad == 0 && c0 + lane < p.n)
+            e.ssq_out[(size_t)tile * SSQ_PITCH + c0 + lane] =
+                (sm->ssq_part[grp][0][lane] + sm->ssq_part[grp][1][lane]) + (sm->ssq_part[grp][2][lane] + sm->ssq_part[grp][3][lane]);
+        grp_bar(grp);
+        return;
+    }
     if (e.mode == EPI_RAW || e.mode == EPI_RESID) {
         const int f = tile * TILE_M + row;
         if (f < p.m) {
@@ -111,6 +169,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
     }
     // EPI_ROPE_KV: output features [0,d) = q, [d,2d) = k, [2d,3d) = v; tiles never straddle sections
     const int d = e.d_model, dh = e.d_head, half = dh >> 1;
+    const int kv_len = resolve_kv_len(e.kv_len, e.kv_len_dev, e.max_kv_len, p.n);
     const int f = tile * TILE_M + row;
     const int section = f / d, el = f - section * d;
     const int head = el / dh, idx = el - head * dh;
@@ -138,7 +197,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
         __half* dst;
         size_t pitch;
         if (section == 0) { dst = (__half*)e.out_t + (size_t)c0 * d + el; pitch = (size_t)d; }
-        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + e.kv_len + c0) * dh + idx; pitch = (size_t)dh; }
+        else { dst = (__half*)e.k_cache + ((size_t)head * e.max_kv_len + kv_len + c0) * dh + idx; pitch = (size_t)dh; }
 #pragma unroll
         for (int j = 0; j < 32; ++j)
             if (c0 + j < p.n) dst[(size_t)j * pitch] = __float2half_rn(v[j]);
@@ -147,7 +206,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, Smem* sm, in
         for (int j = 0; j < 32; ++j) {
             const int node = c0 + j;
             if (node < p.n)
-                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + e.kv_len + node) * dh + idx] = __float2half_rn(v[j]);
+                ((__half*)e.v_cache)[((size_t)head * e.max_kv_len + kv_len + node) * dh + idx] = __float2half_rn(v[j]);
         }
     }
 }

@@ -23,7 +23,9 @@ size_t carve_workspace(ghd_ctx* c, char* base) {
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return base ? base + at : nullptr; };
     const size_t raw_cols = (3 * d > 2 * f) ? 3 * d : 2 * f;
     c->status = (int*)take(256);
+    c->kv_len_word = c->status ? c->status + 16 : nullptr;       // same 256-byte block, its own 64-byte line
     c->counters = (int*)take(sizeof(int) * 4096);
+    for (int b = 0; b < 2; ++b) c->ssq[b] = (float*)take(sizeof(float) * SSQ_MAX_TILES * SSQ_PITCH);
     c->xres = (float*)take(N * d * 4);
     c->hbuf = take(N * d * es);
     c->qbuf = take(N * d * es);
@@ -53,6 +55,7 @@ static ghd_status check_cuda(ghd_ctx* c, const char* where) {
 static ghd_status check_tree(ghd_ctx* c, const ghd_tree* t) {
     if (!t || !t->mask || !t->depth || !t->pos || !t->rope) return fail(c, GHD_EINVAL, "tree: null pointer");
     if (t->n < 1 || t->n > c->cfg.max_nodes || t->n_words != (t->n + 63) / 64) return fail(c, GHD_ETREE, "tree: not built");
+    if (t->kv_len == GHD_KV_LEN_DEVICE) return GHD_OK;       // checked on the device when the tree was built
     if (t->kv_len < 0 || t->kv_len + t->n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: kv_len + n > max_kv_len");
     return GHD_OK;
 }
@@ -112,7 +115,7 @@ static ghd_status attention(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, c
 
 static EpiArgs epi_base(ghd_ctx* c, const ghd_tree* t) {
     EpiArgs e{};
-    e.rope = t->rope; e.kv_len = t->kv_len; e.max_kv_len = c->cfg.max_kv_len; e.d_head = c->cfg.d_head; e.d_model = c->cfg.d_model;
+    e.rope = t->rope; e.kv_len = t->kv_len; e.kv_len_dev = kv_len_dev_of(c, t); e.max_kv_len = c->cfg.max_kv_len; e.d_head = c->cfg.d_head; e.d_model = c->cfg.d_model;
     return e;
 }
 
@@ -133,6 +136,62 @@ static ghd_status layer_body(ghd_ctx* c, const ghd_layer_weights* w, const ghd_k
     return GHD_OK;
 }
 
+// True when the four projections of a layer can run on the tcgen05 path with the norms folded into their
+// epilogues: the projection into the residual stream adds, writes the gain-weighted rows of the next
+// norm and per-tile sums of squares; the projection that reads those rows multiplies by 1 / rms.
+static bool fused_norm_ok(const ghd_ctx* c, int n) {
+    const ghd_model_cfg& m = c->cfg;
+    if (c->opt_fused_norm != 1 || m.dtype != GHD_F16 || c->opt_gemm_path == 1) return false;
+    return gemm_tc_supported(c, n, m.d_model, 3 * m.d_model, EPI_ROPE_KV) && gemm_tc_supported(c, n, m.d_model, m.d_model, EPI_RESID_NORM) &&
+           gemm_tc_supported(c, n, m.d_model, 2 * m.d_ffn, EPI_SWIGLU) && gemm_tc_supported(c, n, m.d_ffn, m.d_model, EPI_RESID_NORM);
+}
+
+static void with_row_scale(ghd_ctx* c, EpiArgs& e) {
+    e.ssq_in = c->ssq[c->h_ssq];
+    e.ssq_in_tiles = c->ssq_tiles[c->h_ssq];
+    e.rms_eps = c->cfg.rms_eps;
+}
+
+// First norm of a call on the fused-norm path.
+static void prenorm_into_h(ghd_ctx* c, const void* gain, int n) {
+    launch_prenorm(c, gain, n, c->hbuf, c->ssq[0]);
+    c->ssq_tiles[0] = 1;
+    c->h_ssq = 0;
+}
+
+// One layer on the fused-norm path.  On entry hbuf holds xres * rms1 gain with its sums of squares in
+// ssq[h_ssq]; on exit hbuf holds xres * next_gain likewise (next_gain = nullptr: residual stream only).
+static ghd_status layer_body_fused(ghd_ctx* c, const ghd_layer_weights* w, const ghd_kv_layer* kv, const ghd_tree* t, const void* next_gain) {
+    const ghd_model_cfg& m = c->cfg;
+    const int n = t->n, d = m.d_model, f = m.d_ffn;
+    ghd_status s;
+    const EpiArgs base = epi_base(c, t);
+    EpiArgs e = base;
+    e.mode = EPI_ROPE_KV; e.out_t = c->qbuf; e.k_cache = kv->k; e.v_cache = kv->v;
+    with_row_scale(c, e);
+    if ((s = project(c, c->hbuf, w->wqkv, n, d, 3 * d, e, t, kv)) != GHD_OK) return s;
+    if ((s = attention(c, c->qbuf, kv, t, c->attnbuf)) != GHD_OK) return s;
+    int nxt = c->h_ssq ^ 1;
+    e = base;
+    e.mode = EPI_RESID_NORM; e.out_f32 = c->xres; e.gain = w->rms2; e.xg_out = c->hbuf; e.ssq_out = c->ssq[nxt];
+    if ((s = project(c, c->attnbuf, w->wo, n, d, d, e, t, kv)) != GHD_OK) return s;
+    c->ssq_tiles[nxt] = d / 128;
+    c->h_ssq = nxt;
+    e = base;
+    e.mode = EPI_SWIGLU; e.out_t = c->ubuf;
+    with_row_scale(c, e);
+    if ((s = project(c, c->hbuf, w->w_gate_up, n, d, 2 * f, e, t, kv)) != GHD_OK) return s;
+    nxt = c->h_ssq ^ 1;
+    e = base;
+    if (next_gain) { e.mode = EPI_RESID_NORM; e.gain = next_gain; e.xg_out = c->hbuf; e.ssq_out = c->ssq[nxt]; }
+    else e.mode = EPI_RESID;
+    e.out_f32 = c->xres;
+    if ((s = project(c, c->ubuf, w->w_down, n, f, d, e, t, kv)) != GHD_OK) return s;
+    if (next_gain) { c->ssq_tiles[nxt] = d / 128; c->h_ssq = nxt; }
+    else c->h_ssq = -1;
+    return GHD_OK;
+}
+
 static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer* kv, const ghd_tree* t,
                             const int32_t* tokens, float* logits, int32_t* amax) {
     const ghd_model_cfg& m = c->cfg;
@@ -140,6 +199,16 @@ static ghd_status step_body(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer
     launch_embed(c, w->embed, tokens, t->n);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = logits;
+    c->h_ssq = -1;
+    if (fused_norm_ok(c, t->n) && gemm_tc_supported(c, t->n, m.d_model, m.vocab, EPI_RAW)) {
+        prenorm_into_h(c, m.n_layers > 0 ? w->layers[0].rms1 : w->rms_final, t->n);
+        for (int l = 0; l < m.n_layers; ++l)
+            if ((s = layer_body_fused(c, &w->layers[l], &kv[l], t, l + 1 < m.n_layers ? w->layers[l + 1].rms1 : w->rms_final)) != GHD_OK) return s;
+        with_row_scale(c, e);       // hbuf stays gain-weighted: the drafting heads divide by the rms themselves
+        if ((s = project(c, c->hbuf, w->lm_head, t->n, m.d_model, m.vocab, e, t, nullptr)) != GHD_OK) return s;
+        launch_argmax(c, logits, t->n, m.vocab, amax);
+        return GHD_OK;
+    }
     for (int l = 0; l < m.n_layers; ++l)
         if ((s = layer_body(c, &w->layers[l], &kv[l], t)) != GHD_OK) return s;
     norm_into_h(c, w->rms_final, t->n);
@@ -176,11 +245,13 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = c->opt_chain_calls = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = c->opt_chain_calls = c->opt_fused_norm = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
     c->pending.active = 0;
+    c->h_ssq = -1;
+    c->kv_len_hint = 0;
     c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     c->attr_gemm = c->attr_attn = false;
     c->launches = 0;
@@ -230,6 +301,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_NO_PDL: c->opt_no_pdl = value ? 1 : 0; break;
         case GHD_OPT_GEMM_STAGES: if (value == 1 || value > 10) return GHD_EINVAL; c->opt_gemm_stages = value; break;
         case GHD_OPT_CHAIN_CALLS: c->opt_chain_calls = value ? 1 : 0; break;
+        case GHD_OPT_FUSED_NORM: if (value > 1) return GHD_EINVAL; c->opt_fused_norm = value; break;
         case GHD_OPT_ATTN_SPARSE: if (value > 1) return GHD_EINVAL; c->opt_attn_sparse = value; break;
         case GHD_OPT_GEMM_EPI: if (value > 2) return GHD_EINVAL; c->opt_gemm_epi = value; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
@@ -243,6 +315,10 @@ static ghd_status tree_common(ghd_ctx* c, int32_t n, int32_t kv_len, ghd_tree* t
     if (!tree->mask || !tree->parent || !tree->depth || !tree->pos || !tree->rope) return fail(c, GHD_EINVAL, "tree: null buffer");
     if ((tree->coo_ptr == nullptr) != (tree->coo_col == nullptr)) return fail(c, GHD_EINVAL, "tree: give both index buffers or neither");
     if (n < 1 || n > c->cfg.max_nodes) return fail(c, GHD_ETREE, "tree: n outside [1, max_nodes]");
+    if (kv_len == GHD_KV_LEN_DEVICE) {
+        if (n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: n > max_kv_len");
+        return GHD_OK;
+    }
     if (kv_len < 0) return fail(c, GHD_EINVAL, "tree: negative kv_len");
     if ((int64_t)kv_len + n > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "tree: kv_len + n > max_kv_len");
     return GHD_OK;
@@ -298,6 +374,13 @@ ghd_status ghd_verify_layer(ghd_ctx* c, const ghd_layer_weights* w, ghd_kv_layer
     c->pending.active = 0;
     c->entry_fresh = c->opt_chain_calls ? 0 : 1;
     launch_load_x(c, x_in, tree->n);
+    c->h_ssq = -1;
+    if (fused_norm_ok(c, tree->n)) {
+        prenorm_into_h(c, w->rms1, tree->n);
+        if ((s = layer_body_fused(c, w, kv, tree, nullptr)) != GHD_OK) return s;
+        launch_store_x(c, x_out, tree->n);
+        return check_cuda(c, "verify_layer");
+    }
     if ((s = layer_body(c, w, kv, tree)) != GHD_OK) return s;
     if (c->pending.active) launch_fold_pending(c, tree->n, nullptr, nullptr, x_out);
     else launch_store_x(c, x_out, tree->n);
@@ -331,7 +414,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope); push(tree->coo_ptr); push(tree->coo_col);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
-    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse, c->opt_chain_calls})
+    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse, c->opt_chain_calls, c->opt_fused_norm})
         key.push_back((uint64_t)(uint32_t)o);       // every option that changes what is enqueued
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];
@@ -386,9 +469,26 @@ ghd_status ghd_accept(ghd_ctx* c, const ghd_tree* tree, const int32_t* tokens_de
     return check_cuda(c, "accept");
 }
 
+ghd_status ghd_kv_len_set(ghd_ctx* c, int32_t kv_len) {
+    if (!c) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (kv_len < 0 || kv_len >= c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "kv_len_set: kv_len outside the cache");
+    launch_kv_len_set(c, kv_len);
+    return check_cuda(c, "kv_len_set");
+}
+
+ghd_status ghd_kv_len_get(ghd_ctx* c, int32_t* kv_len_host) {
+    if (!c || !kv_len_host) return GHD_EINVAL;
+    if (!c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return check_cuda(c, "stream synchronize");
+    if (cudaMemcpy(kv_len_host, c->kv_len_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return check_cuda(c, "kv_len read");
+    return GHD_OK;
+}
+
 ghd_status ghd_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int32_t n_layers, int32_t kv_len, const ghd_accept_result* result_dev) {
     if (!c || !kv || !result_dev || n_layers < 1) return GHD_EINVAL;
-    if (kv_len < 0 || kv_len + 1 > c->cfg.max_kv_len) return fail(c, GHD_ENOSPACE, "kv_commit: kv_len outside the cache");
+    if (kv_len == GHD_KV_LEN_DEVICE && !c->ws) return fail(c, GHD_ENOSPACE, "no workspace set");
+    if (kv_len != GHD_KV_LEN_DEVICE && (kv_len < 0 || kv_len + 1 > c->cfg.max_kv_len)) return fail(c, GHD_ENOSPACE, "kv_commit: kv_len outside the cache");
     for (int l = 0; l < n_layers; ++l)
         if (!kv[l].k || !kv[l].v) return fail(c, GHD_EINVAL, "kv_commit: null cache pointer");
     launch_kv_commit(c, kv, n_layers, kv_len, result_dev);
@@ -410,7 +510,7 @@ ghd_status ghd_medusa_draft(ghd_ctx* c, const ghd_medusa_weights* w, const ghd_a
     float* logits = logits_dev ? logits_dev : c->mlogits;
     c->pending.active = 0;
     c->entry_fresh = c->opt_chain_calls ? 0 : 1;
-    launch_medusa_gather(c, result_dev, c->attnbuf);
+    launch_medusa_gather(c, result_dev, c->attnbuf, c->h_ssq >= 0 ? c->ssq[c->h_ssq] : nullptr, c->h_ssq >= 0 ? c->ssq_tiles[c->h_ssq] : 0);
     EpiArgs e{};
     e.mode = EPI_RAW; e.out_f32 = c->raw;
     ghd_status s = project(c, c->attnbuf, w->w1, 1, d, K * d, e, nullptr, nullptr);      // all heads' W1 rows in one projection
@@ -489,9 +589,17 @@ ghd_status ghd_sync_status(ghd_ctx* c) {
     if (!c->ws) return GHD_OK;
     int st = 0;
     if (cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return check_cuda(c, "status read");
+    if (st == DEV_KV_RANGE) {
+        snprintf(c->err, sizeof(c->err), "the cache length on the device left [0, max_kv_len - n]");
+        cudaMemset(c->status, 0, sizeof(int));
+        return GHD_ENOSPACE;
+    }
     if (st != DEV_OK) {
         snprintf(c->err, sizeof(c->err), "device wait expired (code %d)", st);
+        int keep = 0;                                          // the cache length survives the clean-up
+        cudaMemcpy(&keep, c->kv_len_word, sizeof(int), cudaMemcpyDeviceToHost);
         cudaMemset(c->status, 0, 256 + sizeof(int) * 4096);   // status word and tile arrival counters
+        cudaMemcpy(c->kv_len_word, &keep, sizeof(int), cudaMemcpyHostToDevice);
         return GHD_ETIMEOUT;
     }
     return GHD_OK;

@@ -15,7 +15,7 @@
 namespace ghd {
 
 // Device status word values (first failure wins).
-enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_TIMEOUT_TMEM = 4, DEV_TIMEOUT_GRID = 5 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPI = 3, DEV_TIMEOUT_TMEM = 4, DEV_TIMEOUT_GRID = 5, DEV_KV_RANGE = 6 };
 
 // Epilogues of the projection GEMMs.
 enum Epilogue : int {
@@ -24,7 +24,11 @@ enum Epilogue : int {
     EPI_RESID = 2,    // xres[n][m] += acc (float residual stream)
     EPI_SWIGLU = 3,   // u T [n][m/2] = SiLU(gate) * up, weight rows [gate | up]
     EPI_DEFER = 4,    // partial tiles only; the next kernel adds them to the residual stream
+    EPI_RESID_NORM = 5,   // xres += acc; xg T [n][m] = xres * gain (not yet divided by the rms); per-tile sums of squares
 };
+
+constexpr int SSQ_PITCH = GHD_MAX_NODES;   // floats per 128-feature tile in a sum-of-squares buffer
+constexpr int SSQ_MAX_TILES = 64;
 
 struct EpiArgs {
     int mode;
@@ -34,6 +38,16 @@ struct EpiArgs {
     void* v_cache;
     const float* rope;    // [n][d_head] cos/sin pairs
     int kv_len, max_kv_len, d_head, d_model;
+    const int* kv_len_dev;    // non-null: the cache length comes from this device word instead of kv_len
+    // Column scale: the input rows are gain-weighted but not yet normalised; node i's result is multiplied by
+    // 1 / sqrt(sum_t ssq_in[t][i] / k + eps) before the epilogue proper (nullptr: no scale).
+    const float* ssq_in;
+    int ssq_in_tiles;
+    float rms_eps;
+    // EPI_RESID_NORM (out_f32 = residual stream): gain T [m] of the NEXT norm, xg_out T [n][m], ssq_out [m/128][SSQ_PITCH]
+    const void* gain;
+    void* xg_out;
+    float* ssq_out;
 };
 
 struct TmapKey {
@@ -68,7 +82,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -82,9 +96,14 @@ struct ghd_ctx {
     float* att_ml;    // float [splits][max_nodes][n_heads][2] running max / sum
     float* gemm_part; // float [ctas][2][256][128] split tile partial sums
     int* counters;    // int [tiles] arrival counters (zero between launches)
+    float* ssq[2];    // float [SSQ_MAX_TILES][SSQ_PITCH] per-tile sums of squares of the residual stream (two, used in turn)
+    int ssq_tiles[2]; // tiles that hold data in each
+    int h_ssq;        // which of them describes hbuf (-1: hbuf is already normalised)
     float* logits;    // float [max_nodes][vocab]
     float* mlogits;   // float [8][vocab] logits of the drafting heads
     int* status;      // device status word
+    int* kv_len_word; // device word with the cache length (calls given GHD_KV_LEN_DEVICE read it)
+    int kv_len_hint;  // what the host last wrote there: sizes launches whose grid depends on the length
     int max_splits;
     ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
@@ -106,6 +125,14 @@ namespace ghd {
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// Cache length of a call: the host's value, or (dev != nullptr) the context's device word, clamped so that the
+// rows kv_len .. kv_len + n - 1 stay inside the cache whatever the word holds.
+__device__ __forceinline__ int resolve_kv_len(int host, const int* dev, int max_kv_len, int n) {
+    if (!dev) return host;
+    int v = __ldcg(dev);
+    if (v > max_kv_len - n) v = max_kv_len - n;
+    return v < 0 ? 0 : v;
+}
 #endif
 
 // cluster_x > 1: the CTAs of a grid row (gridDim.x a multiple of cluster_x) are launched as thread-block clusters.
@@ -154,6 +181,8 @@ void launch_load_x(ghd_ctx* c, const void* x_in, int n);     // T [n][d] -> xres
 void launch_store_x(ghd_ctx* c, void* x_out, int n);         // xres -> T [n][d]
 void launch_embed(ghd_ctx* c, const void* embed, const int32_t* tokens, int n);
 void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out);
+// xg T [n][d] = xres * g (not normalised), ssq[0][node] = sum of squares of the row
+void launch_prenorm(ghd_ctx* c, const void* g, int n, void* xg, float* ssq);
 // xres += sum of the pending partial tiles; then optionally h = RMSNorm(xres) * g and/or x_out = T(xres)
 void launch_fold_pending(ghd_ctx* c, int n, const void* g, void* h_out, void* x_out);
 void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, const ghd_kv_layer* kv);
@@ -162,11 +191,18 @@ void launch_residual(ghd_ctx* c, const float* proj_raw, int n);
 void launch_argmax(ghd_ctx* c, const float* logits, int n, int v, int32_t* out);
 void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const int32_t* amax, ghd_accept_result* out);
 // drafting heads (kernels_small.cu)
-void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel);                 // h_sel T [d] = hbuf[last accepted node]
+// h_sel T [d] = hbuf[last accepted node], divided by the row's rms when hbuf is not yet normalised (ssq != nullptr)
+void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel, const float* ssq, int ssq_tiles);
 void launch_medusa_res(ghd_ctx* c, const void* h_sel, const float* raw, int heads, void* y);        // y T [heads][d] = h + SiLU(raw)
 void launch_medusa_topk(ghd_ctx* c, const float* logits, int heads, int vocab, const int* topk, int32_t* cand);
 void launch_tree_fill(ghd_ctx* c, const int32_t* cand, const ghd_accept_result* res, const int32_t* level, const int32_t* rank, int n, int32_t* tokens);
+// kv_len < 0: rows relative to the device word, which a second kernel then advances by n_matched + 1
 void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_len, const ghd_accept_result* res);
+void launch_kv_len_set(ghd_ctx* c, int kv_len);
+// the device word when the tree's length is GHD_KV_LEN_DEVICE, else nullptr
+inline const int* kv_len_dev_of(const ghd_ctx* c, const ghd_tree* t) { return t->kv_len < 0 ? c->kv_len_word : nullptr; }
+// the length launch geometry is sized for
+inline int kv_len_host_of(const ghd_ctx* c, const ghd_tree* t) { return t->kv_len < 0 ? c->kv_len_hint : t->kv_len; }
 
 // gemm_simt.cu : y float [n][m] = x T [n][k] * w T [m][k]^T
 void launch_gemm_simt(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, float* y);

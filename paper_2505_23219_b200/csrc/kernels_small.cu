@@ -25,10 +25,21 @@ struct CooPtrArg { uint16_t ptr[GHD_MAX_NODES + 1]; };
 // the slow part (pow and sincos in double), hence several blocks.
 constexpr int TREE_NODES_PER_BLOCK = 8;
 
+// Length of the cache for a tree kernel: the host's value, or the device word (clamped into the cache; a word
+// outside [0, max_kv_len - n] is recorded in the status word by the kernel's first thread).
+__device__ __forceinline__ int tree_kv_len(int host, const int* dev, int max_kv_len, int n, int* status, bool reporter) {
+    if (dev && reporter) {
+        const int raw = __ldcg(dev);
+        if (raw < 0 || raw > max_kv_len - n) atomicCAS(status, DEV_OK, DEV_KV_RANGE);
+    }
+    return resolve_kv_len(host, dev, max_kv_len, n);
+}
+
 __global__ void k_tree_build(ParentArg pa, CooPtrArg cp, int n, int n_words, int kv_len, int d_head, double theta,
                              uint64_t* mask, int32_t* parent, int32_t* depth, int32_t* pos, float* rope,
-                             int32_t* coo_ptr, int32_t* coo_col) {
+                             int32_t* coo_ptr, int32_t* coo_col, const int* kv_len_dev, int max_kv_len, int* status) {
     __shared__ int spos[TREE_NODES_PER_BLOCK];
+    kv_len = tree_kv_len(kv_len, kv_len_dev, max_kv_len, n, status, blockIdx.x == 0 && threadIdx.x == 0);
     const int first = blockIdx.x * TREE_NODES_PER_BLOCK;
     if (threadIdx.x < TREE_NODES_PER_BLOCK) {
         const int i = first + threadIdx.x;
@@ -67,8 +78,10 @@ __global__ void k_tree_build(ParentArg pa, CooPtrArg cp, int n, int n_words, int
 
 // Explicit-mask variant: mask (and optionally depth, parent) were copied in.
 __global__ void k_tree_from_mask(CooPtrArg cp, int n, int n_words, int kv_len, int d_head, double theta, int have_depth,
-                                 const uint64_t* mask, int32_t* depth, int32_t* pos, float* rope, int32_t* coo_ptr, int32_t* coo_col) {
+                                 const uint64_t* mask, int32_t* depth, int32_t* pos, float* rope, int32_t* coo_ptr, int32_t* coo_col,
+                                 const int* kv_len_dev, int max_kv_len, int* status) {
     const int i = threadIdx.x;
+    kv_len = tree_kv_len(kv_len, kv_len_dev, max_kv_len, n, status, threadIdx.x == 0);
     if (i < n && coo_ptr) {
         coo_ptr[i] = cp.ptr[i];
         if (i == n - 1) coo_ptr[n] = cp.ptr[n];
@@ -116,7 +129,7 @@ void launch_tree_build(ghd_ctx* c, const int32_t* parent_host, ghd_tree* t) {
     t->nnz = cp.ptr[t->n];
     k_tree_build<<<(t->n + TREE_NODES_PER_BLOCK - 1) / TREE_NODES_PER_BLOCK, 256, 0, c->cur>>>(pa, cp, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                      (double)c->cfg.rope_theta, t->mask, t->parent, t->depth,
-                                                     t->pos, t->rope, t->coo_ptr, t->coo_col);
+                                                     t->pos, t->rope, t->coo_ptr, t->coo_col, kv_len_dev_of(c, t), c->cfg.max_kv_len, c->status);
     c->launches++;
 }
 
@@ -132,7 +145,8 @@ void launch_tree_from_mask(ghd_ctx* c, ghd_tree* t, bool have_depth, const uint6
     t->nnz = cp.ptr[t->n];
     k_tree_from_mask<<<1, GHD_MAX_NODES, 0, c->cur>>>(cp, t->n, t->n_words, t->kv_len, c->cfg.d_head,
                                                          (double)c->cfg.rope_theta, have_depth ? 1 : 0, t->mask,
-                                                         t->depth, t->pos, t->rope, t->coo_ptr, t->coo_col);
+                                                         t->depth, t->pos, t->rope, t->coo_ptr, t->coo_col, kv_len_dev_of(c, t),
+                                                         c->cfg.max_kv_len, c->status);
     c->launches++;
 }
 
@@ -269,6 +283,34 @@ void launch_rmsnorm(ghd_ctx* c, const float* x, const void* g, int n, void* out)
                    launch_k(c, true, k_rmsnorm<__half>, n, threads, 0, x, (const __half*)g, (__half*)out, d, c->cfg.rms_eps));
 }
 
+// The first norm of a call when the projections normalise in their epilogues: xg = x * g (gain-weighted,
+// not divided by the rms) and the row's sum of squares as the single "tile" of a sum-of-squares buffer.
+__global__ void __launch_bounds__(1024) k_prenorm(const float* __restrict__ x, const __half* __restrict__ g, __half* __restrict__ xg,
+                                                  float* __restrict__ ssq, int d) {
+    __shared__ float red[32];
+    pdl_wait();
+    pdl_trigger();
+    const float* row = x + (size_t)blockIdx.x * d;
+    __half* orow = xg + (size_t)blockIdx.x * d;
+    const int nv = d >> 2;
+    float ss = 0.f;
+    for (int idx = threadIdx.x; idx < nv; idx += blockDim.x) {
+        const float4 w = *reinterpret_cast<const float4*>(row + 4 * idx);
+        const float4 gg = load4<__half>(g + 4 * idx);
+        ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+        store4<__half>(orow + 4 * idx, w.x * gg.x, w.y * gg.y, w.z * gg.z, w.w * gg.w);
+    }
+    ss = block_sum(ss, red);
+    if (threadIdx.x == 0) ssq[blockIdx.x] = ss;
+}
+
+void launch_prenorm(ghd_ctx* c, const void* g, int n, void* xg, float* ssq) {
+    const int d = c->cfg.d_model;
+    int threads = ((d / 4 + 31) / 32) * 32;
+    if (threads > 1024) threads = 1024;
+    launch_k(c, true, k_prenorm, n, threads, 0, (const float*)c->xres, (const __half*)g, (__half*)xg, ssq, d);
+}
+
 // Folds the partial tiles of a deferred-reduction projection into the residual stream and,
 // in the same pass, produces the next RMSNorm output.  One block per node; a thread owns four
 // consecutive features (all inside one 128-row tile), adds that tile's contributors in CTA
@@ -347,7 +389,9 @@ void launch_fold_pending(ghd_ctx* c, int n, const void* g, void* h_out, void* x_
 // (t, t + dh/2), writes q to the query buffer and k, v to cache row kv_len + node.
 template <typename T>
 __global__ void k_rope_append(const float* __restrict__ qkv, const float* __restrict__ rope, T* __restrict__ q,
-                              T* __restrict__ kc, T* __restrict__ vc, int n, int heads, int dh, int kv_len, int max_kv) {
+                              T* __restrict__ kc, T* __restrict__ vc, int n, int heads, int dh, int kv_len, int max_kv,
+                              const int* __restrict__ kv_len_dev) {
+    kv_len = resolve_kv_len(kv_len, kv_len_dev, max_kv, n);
     const int half = dh / 2, d = heads * dh;
     const size_t total = (size_t)n * heads * half;
     for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
@@ -373,9 +417,9 @@ void launch_rope_append(ghd_ctx* c, const float* qkv_raw, const ghd_tree* t, con
     const int g = grid_for(total, 256, 8 * c->sm_count);
     GHD_DISPATCH_T(c,
         (k_rope_append<float><<<g, 256, 0, c->cur>>>(qkv_raw, t->rope, (float*)c->qbuf, (float*)kv->k, (float*)kv->v,
-                                                         t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)),
+                                                         t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len, kv_len_dev_of(c, t))),
         (k_rope_append<__half><<<g, 256, 0, c->cur>>>(qkv_raw, t->rope, (__half*)c->qbuf, (__half*)kv->k, (__half*)kv->v,
-                                                          t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len)));
+                                                          t->n, m.n_heads, m.d_head, t->kv_len, m.max_kv_len, kv_len_dev_of(c, t))));
     c->launches++;
 }
 
@@ -510,14 +554,20 @@ void launch_accept(ghd_ctx* c, const ghd_tree* t, const int32_t* tokens, const i
 // ---------------------------------------------------------------- drafting heads
 // h_sel = hidden state (after the final norm) of the last accepted node, picked on the device.
 template <typename T>
-__global__ void k_medusa_gather(const T* __restrict__ hbuf, const ghd_accept_result* __restrict__ res, int d, int max_nodes, T* __restrict__ h_sel) {
+__global__ void k_medusa_gather(const T* __restrict__ hbuf, const ghd_accept_result* __restrict__ res, int d, int max_nodes, T* __restrict__ h_sel,
+                                const float* __restrict__ ssq, int ssq_tiles, float eps) {
     int m = res->n_matched;
     if (m < 0 || m >= GHD_MAX_NODES) m = 0;
     int node = res->nodes[m];
     if (node < 0 || node >= max_nodes) node = 0;
-    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < d; j += gridDim.x * blockDim.x) h_sel[j] = hbuf[(size_t)node * d + j];
+    float r = 1.f;
+    if (ssq) {      // hbuf holds gain-weighted rows that still want their 1 / rms
+        float ss = 0.f;
+        for (int t = 0; t < ssq_tiles; ++t) ss += ssq[(size_t)t * SSQ_PITCH + node];
+        r = rsqrtf(ss / (float)d + eps);
+    }
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < d; j += gridDim.x * blockDim.x) h_sel[j] = (T)((float)hbuf[(size_t)node * d + j] * r);
 }
-
 // y[k][j] = h[j] + SiLU(raw[k * d + j])
 template <typename T>
 __global__ void k_medusa_res(const T* __restrict__ h, const float* __restrict__ raw, int heads, int d, T* __restrict__ y) {
@@ -596,10 +646,11 @@ __global__ void k_tree_fill(const int32_t* __restrict__ cand, const ghd_accept_r
     tokens[i] = (lv >= 1 && lv <= GHD_MAX_DRAFT_HEADS && rk >= 0 && rk < GHD_MAX_TOPK) ? cand[(lv - 1) * GHD_MAX_TOPK + rk] : -1;
 }
 
-void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel) {
+void launch_medusa_gather(ghd_ctx* c, const ghd_accept_result* res, void* h_sel, const float* ssq, int ssq_tiles) {
     const int d = c->cfg.d_model;
-    GHD_DISPATCH_T(c, (k_medusa_gather<float><<<1, 1024, 0, c->cur>>>((const float*)c->hbuf, res, d, c->cfg.max_nodes, (float*)h_sel)),
-                   (k_medusa_gather<__half><<<1, 1024, 0, c->cur>>>((const __half*)c->hbuf, res, d, c->cfg.max_nodes, (__half*)h_sel)));
+    const float eps = c->cfg.rms_eps;
+    GHD_DISPATCH_T(c, (k_medusa_gather<float><<<1, 1024, 0, c->cur>>>((const float*)c->hbuf, res, d, c->cfg.max_nodes, (float*)h_sel, ssq, ssq_tiles, eps)),
+                   (k_medusa_gather<__half><<<1, 1024, 0, c->cur>>>((const __half*)c->hbuf, res, d, c->cfg.max_nodes, (__half*)h_sel, ssq, ssq_tiles, eps)));
     c->launches++;
 }
 
@@ -635,7 +686,8 @@ struct CommitPtrs {
 };
 
 __global__ void k_kv_commit(CommitPtrs ptrs, int heads, int max_kv_len, int row_bytes, int kv_len,
-                            const ghd_accept_result* __restrict__ res) {
+                            const ghd_accept_result* __restrict__ res, const int* __restrict__ kv_len_dev) {
+    kv_len = resolve_kv_len(kv_len, kv_len_dev, max_kv_len, 1);
     const int layer = blockIdx.x / heads, head = blockIdx.x - layer * heads;
     char* base = (char*)(blockIdx.y == 0 ? ptrs.k[layer] : ptrs.v[layer]) + (size_t)head * max_kv_len * row_bytes;
     int m = res->n_matched;
@@ -649,6 +701,18 @@ __global__ void k_kv_commit(CommitPtrs ptrs, int heads, int max_kv_len, int row_
     }
 }
 
+// The cache length after a step: the accepted path adds n_matched + 1 rows (Sec. II-C).
+__global__ void k_kv_len_advance(int* word, const ghd_accept_result* __restrict__ res, int max_kv_len) {
+    int m = res->n_matched;
+    if (m < 0) m = 0;
+    if (m > GHD_MAX_NODES - 1) m = GHD_MAX_NODES - 1;
+    int v = *word;
+    if (v < 0) v = 0;
+    v += m + 1;
+    *word = v > max_kv_len - 1 ? max_kv_len - 1 : v;
+}
+__global__ void k_kv_len_set(int* word, int v) { *word = v; }
+
 void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_len, const ghd_accept_result* res) {
     const ghd_model_cfg& m = c->cfg;
     const int row_bytes = m.d_head * (m.dtype == GHD_F32 ? 4 : 2);
@@ -656,9 +720,21 @@ void launch_kv_commit(ghd_ctx* c, const ghd_kv_layer* kv, int n_layers, int kv_l
         CommitPtrs ptrs{};
         const int cnt = n_layers - l0 < COMMIT_LAYERS ? n_layers - l0 : COMMIT_LAYERS;
         for (int l = 0; l < cnt; ++l) { ptrs.k[l] = kv[l0 + l].k; ptrs.v[l] = kv[l0 + l].v; }
-        k_kv_commit<<<dim3(cnt * m.n_kv_heads, 2), 32, 0, c->cur>>>(ptrs, m.n_kv_heads, m.max_kv_len, row_bytes, kv_len, res);
+        k_kv_commit<<<dim3(cnt * m.n_kv_heads, 2), 32, 0, c->cur>>>(ptrs, m.n_kv_heads, m.max_kv_len, row_bytes, kv_len, res,
+                                                                    kv_len < 0 ? c->kv_len_word : nullptr);
         c->launches++;
     }
+    if (kv_len < 0) {          // every move above read the old length: advance the word behind them
+        k_kv_len_advance<<<1, 1, 0, c->cur>>>(c->kv_len_word, res, m.max_kv_len);
+        c->launches++;
+        if (c->kv_len_hint + 1 < m.max_kv_len) c->kv_len_hint += 1;      // a step emits at least one token
+    }
+}
+
+void launch_kv_len_set(ghd_ctx* c, int kv_len) {
+    k_kv_len_set<<<1, 1, 0, c->cur>>>(c->kv_len_word, kv_len);
+    c->launches++;
+    c->kv_len_hint = kv_len;
 }
 
 }  // namespace ghd

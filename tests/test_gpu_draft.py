@@ -162,3 +162,67 @@ def test_self_drafting_decode_loop_is_lossless(ghd):
         L += m + 1
     ghd.ghd_sync_status(ctx)
     assert out == g[1:len(out) + 1]
+
+
+@pytest.mark.parametrize("shape,graph", [(SMALL32, 0), (SMALL16, 0), (SMALL16, 2)], ids=["f32", "f16", "f16graph"])
+def test_self_drafting_loop_with_the_cache_length_on_the_device(ghd, shape, graph):
+    """The same loop with no host read between steps: the cache length lives in the context's device word, which
+    ghd_kv_commit advances; positions, appended rows and attention follow it.  One read-back at the end."""
+    import torch
+    L0, steps, width = 12, 7, 14
+    acc = [[0.6, 0.3, 0.2, 0.1], [0.5, 0.3, 0.1], [0.4, 0.2]]
+    most = steps * (len(acc) + 1)
+    Lmax = L0 + most + width + 1
+    head = wl.head_weights(shape, 46)
+    layers = [wl.layer_weights(shape, 46, l, random_gains=True) for l in range(shape.n_layers)]
+    fresh = lambda: [wl.kv_cache(shape, 46, l, L0, Lmax) for l in range(shape.n_layers)]
+    o_caches = fresh()
+    g, gaps, first_logits = [5], [], None
+    for s in range(most + 1):
+        vis, _, pos = oracle.tree_build([-1], L0 + s)
+        logits, am = oracle.step(shape, head, layers, o_caches, L0 + s, vis, pos, [g[-1]])
+        first_logits = logits[0].copy() if first_logits is None else first_logits
+        top = np.partition(logits[0], -2)
+        gaps.append(float(top[-1] - top[-2]))
+        g.append(int(am[0]))
+    topk = tuple(len(a) for a in acc)
+    parent, paths, _ = arca.build_tree(acc, width)
+    level = to_dev(np.array([len(p) for p in paths], np.int32))
+    rank = to_dev(np.array([p[-1] if p else 0 for p in paths], np.int32))
+    w1, w2 = _heads(shape, 930, len(acc))
+    mw = ghd.MedusaWeights(to_dev(w1), to_dev(w2))
+    gw = ghd.ModelWeights(to_dev(head["embed"]), [gpu_layer_weights(w) for w in layers], to_dev(head["rms_final"]), to_dev(head["lm_head"]))
+    gkv = [ghd.KvLayer(to_dev(k), to_dev(v), ghd.KV_LEN_DEVICE) for k, v in fresh()]     # every row finite (generated data)
+    ctx = ghd.ghd_create(gpu_cfg(shape, Lmax, width))
+    ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, graph)
+    ghd.ghd_kv_len_set(ctx, L0)
+    tok_d = to_dev(np.array([g[0]] + [0] * (width - 1), np.int32))
+    tree, results = None, []
+    amax = torch.empty(width, dtype=torch.int32, device="cuda")        # fixed buffers: graph mode replays one graph
+    logits_d = torch.empty((width, shape.vocab), dtype=torch.float32, device="cuda")
+    first = None
+    for _ in range(steps):
+        tree = ghd.ghd_tree_build(ctx, parent, ghd.KV_LEN_DEVICE, tree=tree)
+        ghd.ghd_verify_step(ctx, gw, gkv, tree, tok_d, logits=logits_d, argmax=amax)
+        first = logits_d[0].clone() if first is None else first
+        res = ghd.ghd_accept(ctx, tree, tok_d, amax)
+        ghd.ghd_kv_commit(ctx, gkv, ghd.KV_LEN_DEVICE, res)
+        cand = ghd.ghd_medusa_draft(ctx, mw, res, topk)
+        ghd.ghd_tree_fill_tokens(ctx, cand, res, level, rank, tokens=tok_d)
+        results.append(res)
+    L_end = ghd.ghd_kv_len_get(ctx)                            # the only synchronising read
+    ghd.ghd_sync_status(ctx)
+    # token parity needs clear winners: every greedy step's top-1/top-2 gap must dwarf the logit error seen at the root
+    err = np.abs(first.cpu().numpy().astype(np.float64) - first_logits).max()
+    assert err <= tol_for(shape.dtype) * np.abs(first_logits).max()
+    assert min(gaps) > 8.0 * err, "seed gives a near-tie; pick another"
+    out = []
+    for r in torch.stack(results).cpu().numpy():
+        out += [int(t) for t in r[258:259 + int(r[0])]]
+    assert steps <= len(out) <= most and L_end == L0 + len(out)
+    assert out == g[1:len(out) + 1]
+    keep = len(out)
+    tol = tol_for(shape.dtype)
+    for (ok, ov), kv in zip(o_caches, gkv):
+        assert max_rel_err(kv.k.float().cpu().numpy()[:, L0:L0 + keep], ok[:, L0:L0 + keep]) <= tol
+        assert max_rel_err(kv.v.float().cpu().numpy()[:, L0:L0 + keep], ov[:, L0:L0 + keep]) <= tol

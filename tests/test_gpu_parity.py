@@ -84,7 +84,7 @@ def test_argument_errors_launch_nothing(ghd):
     before = ghd.ghd_launch_count(ctx)
     cases = [([0, 0], 0, "GHD_ETREE"), ([-1, 1], 0, "GHD_ETREE"), ([-1, -1], 0, "GHD_ETREE"),
              ([-1] + [0] * 16, 0, "GHD_ETREE"), ([], 0, "GHD_ETREE"), ([-1, 0], 127, "GHD_ENOSPACE"),
-             ([-1, 0], -1, "GHD_EINVAL")]
+             ([-1, 0], -2, "GHD_EINVAL")]      # -1 would be GHD_KV_LEN_DEVICE
     for parent, kv_len, want in cases:
         with pytest.raises(ghd.GhdError) as e:
             ghd.ghd_tree_build(ctx, parent, kv_len)
@@ -176,8 +176,8 @@ def test_linear_tcgen05_path(ghd, n, k, m):
         assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
 
 
-def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0):
-    Lmax = L + n + 3
+def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0, on_device=False):
+    Lmax = L + n + (150 if on_device else 3)               # on_device: the kernels see cache rows far past kv_len + n
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
     if path:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_PATH, path)
@@ -192,6 +192,9 @@ def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0
     k_new = kc[:, L:L + n].transpose(1, 0, 2)
     v_new = vc[:, L:L + n].transpose(1, 0, 2)
     want = oracle.tree_attention(q, k_new, v_new, kc, vc, L, vis)
+    if on_device:                                           # the length comes from the context's device word
+        ghd.ghd_kv_len_set(ctx, L)
+        L = ghd.KV_LEN_DEVICE
     tree = ghd.ghd_tree_build(ctx, parent, L)
     out = ghd.ghd_tree_attention(ctx, to_dev(q.reshape(n, H * dh)), ghd.KvLayer(to_dev(kc), to_dev(vc), L), tree)
     ghd.ghd_sync_status(ctx)
@@ -221,6 +224,19 @@ def test_tree_attention_sparse_part_from_the_coordinate_index(ghd, shape, n, L, 
     assert err <= (2e-5 if shape.dtype == "f32" else 2e-3)
     if shape.dtype == "f16":
         assert _attention_case(ghd, shape, n, L, parent, splits, path=1, sparse=1) <= 2e-3      # cache part on CUDA cores
+
+
+@pytest.mark.parametrize("shape", [SMALL32, SMALL16, SMALL16_DH128], ids=["f32", "f16", "f16dh128"])
+@pytest.mark.parametrize("n,L,splits", ATTN_CASES + [(64, 2048, 0), (200, 1000, 7)])
+def test_tree_attention_with_the_cache_length_on_the_device(ghd, shape, n, L, splits):
+    """GHD_KV_LEN_DEVICE: the kernels read the length from the device word; the cache buffers are longer than
+    kv_len + n and every row of them holds (finite) data that must not leak into the result."""
+    parent = wl.random_tree(n, 8, 1000 + n, max_children=6)
+    tol = 2e-5 if shape.dtype == "f32" else 2e-3
+    assert _attention_case(ghd, shape, n, L, parent, splits, on_device=True) <= tol
+    assert _attention_case(ghd, shape, n, L, parent, splits, sparse=1, on_device=True) <= tol
+    if shape.dtype == "f16":
+        assert _attention_case(ghd, shape, n, L, parent, splits, path=1, on_device=True) <= tol
 
 
 @pytest.mark.parametrize("n,L,splits", [(64, 2048, 0), (64, 2048, 5), (200, 1000, 0), (256, 4096, 0), (49, 640, 3)])
@@ -387,6 +403,19 @@ def test_small_layers_forced_tcgen05_gemm(ghd, n, L):
                 opts=[(g.OPT_GEMM_PATH, 2)])
 
 
+@pytest.mark.parametrize("n,L", [(1, 40), (13, 100), (64, 77), (256, 31)])
+def test_small_layers_with_the_norms_in_the_projection_epilogues(ghd, n, L):
+    """RMSNorm as (gain-weighted rows + per-tile sums of squares) out of one projection and a 1 / rms column scale in the next."""
+    import paper_2505_23219_b200 as g
+    ctx = _layer_case(ghd, SMALL16_DH128, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6), opts=[(g.OPT_FUSED_NORM, 1)])
+    assert ghd.ghd_path_count(ctx, ghd.PATH_GEMM_TILE) >= 4
+
+
+def test_config2_llama7b_layer_f16_with_the_norms_in_the_projection_epilogues(ghd):
+    import paper_2505_23219_b200 as g
+    _layer_case(ghd, wl.LLAMA7B, 2, 64, 1024, wl.medusa_tree(64), gains=False, opts=[(g.OPT_FUSED_NORM, 1)])
+
+
 def test_config2_llama7b_layer_f16(ghd):
     """LLaMA-7B-shaped layer, half weights, KV 1024, 64-node Medusa-style tree."""
     _layer_case(ghd, wl.LLAMA7B, 2, 64, 1024, wl.medusa_tree(64), gains=False)
@@ -465,8 +494,8 @@ def _model(ghd, shape, config_id, L, Lmax):
     return head, layers, caches, gw, gkv
 
 
-@pytest.mark.parametrize("shape,graph", [(SMALL32, 0), (SMALL16, 0), (SMALL16, 2), (SMALL16_DH128, 0), (SMALL16_DH128, 2)],
-                         ids=["f32", "f16", "f16graph", "f16dh128", "f16dh128graph"])
+@pytest.mark.parametrize("shape,graph", [(SMALL32, 0), (SMALL16, 0), (SMALL16, 2), (SMALL16_DH128, 0), (SMALL16_DH128, 2), (SMALL16_DH128, -1)],
+                         ids=["f32", "f16", "f16graph", "f16dh128", "f16dh128graph", "f16dh128-norms-in-epilogues"])
 def test_small_step_logits_argmax_accept(ghd, shape, graph):
     n, L = 24, 90
     Lmax = L + n
@@ -481,6 +510,9 @@ def test_small_step_logits_argmax_accept(ghd, shape, graph):
     want_logits, want_amax = oracle.step(shape, head, layers, [wl.kv_cache(shape, 13, l, L, Lmax) for l in range(shape.n_layers)],
                                          L, vis, pos, tokens)
     ctx = make_ctx(ghd, shape, Lmax, n)
+    if graph < 0:
+        graph = 0
+        ghd.ghd_set_option(ctx, ghd.OPT_FUSED_NORM, 1)
     ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, graph)
     tree = ghd.ghd_tree_build(ctx, parent, L)
     tok_d = to_dev(tokens)
