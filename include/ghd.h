@@ -68,6 +68,9 @@ typedef enum ghd_option {
                                  the residual stream leaves gain-weighted rows and per-tile sums of squares, its
                                  consumer multiplies by 1 / rms); 0 = separate reduction + norm kernels (default:
                                  faster as measured, the split tiles of the narrow projections finish in parallel)  */
+    GHD_OPT_GEMM_PAIR = 12,   /* tcgen05 GEMM on clusters of two CTAs (cta_group::2: a pair shares the activation slab of
+                                 two neighbouring weight tiles, each CTA loading half of it): 0 = for trees of more
+                                 than 128 nodes, 1 = never, 2 = whenever the shape allows (even tile count)          */
     GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
                                  Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
                                  nobody sees them (default); 1 = per-query list of visible nodes (the
@@ -175,7 +178,8 @@ typedef enum ghd_path {
     GHD_PATH_GEMM_SIMT = 1,   /* CUDA-core projection                                 */
     GHD_PATH_ATTN_TC = 2,     /* tcgen05 tree attention                               */
     GHD_PATH_ATTN_SIMT = 3,   /* CUDA-core tree attention                             */
-    GHD_PATH_ATTN_COO = 4     /* sparse part gathered from the coordinate index        */
+    GHD_PATH_ATTN_COO = 4,    /* sparse part gathered from the coordinate index        */
+    GHD_PATH_GEMM_PAIR = 5    /* tcgen05 projection on CTA pairs (counted besides GEMM_TILE) */
 } ghd_path;
 int64_t ghd_path_count(const ghd_ctx *ctx, int32_t path);
 

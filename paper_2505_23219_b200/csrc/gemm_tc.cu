@@ -39,25 +39,49 @@ namespace {
 // TWO: eight epilogue warps in two groups (trees of more than 32 nodes: several 32-column chunks per tile);
 // otherwise four epilogue warps, which a single chunk cannot keep more of busy and which leaves each thread
 // the full register budget.
-template <bool TWO>
+// PAIR: the grid is made of clusters of two CTAs that work on two neighbouring 128-row weight tiles at once
+// (tcgen05 cta_group::2, MMA M = 256): each CTA loads its own weight tile but only HALF of the activation rows;
+// one thread of the even CTA issues the MMAs, which read both CTAs' shared memory and fill both CTAs' tensor
+// memory.  A wide tree's activation slab (up to 32 KB per 64-wide k-step against 16 KB of weights) is then
+// fetched once per 256 weight rows instead of once per 128.  Every CTA issues its own plain TMA loads (no
+// multicast); the pair shares the ring's "full" barriers in the even CTA.  Work units ("wt") are tile pairs dealt to
+// clusters; each CTA runs the epilogue of its own tile exactly as in the single-CTA kernel.
+template <bool TWO, bool PAIR>
 __global__ void __launch_bounds__(TWO ? THREADS_TC : THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t* tiles = smem_raw + pad;
-    const uint32_t a_slab = TILE_M * TILE_K * 2, b_slab = (uint32_t)p.nb * TILE_K * 2;
+    const int nb_cta = PAIR ? p.nb / 2 : p.nb;              // activation rows this CTA loads
+    const uint32_t a_slab = TILE_M * TILE_K * 2, b_slab = (uint32_t)nb_cta * TILE_K * 2;
     const uint32_t a_bytes = p.ks * a_slab, b_bytes = p.ks * b_slab;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     Smem* sm = reinterpret_cast<Smem*>(tiles + (size_t)p.stages * stage_bytes);
     const uint32_t tiles_addr = smem_u32(tiles);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, cta = blockIdx.x;
-    const long long total = (long long)p.n_tiles * p.kiters;
-    const long long it_beg = total * cta / G, it_end = total * (cta + 1) / G;
+    const int cta = blockIdx.x;
+    const int rank = PAIR ? (int)cluster_ctarank() : 0;      // 0: the CTA that issues the pair's MMAs
+    const int G = PAIR ? gridDim.x / 2 : gridDim.x, wk = PAIR ? cta >> 1 : cta;     // workers and this CTA's worker
+    const long long total = (long long)p.n_work * p.kiters;
+    const long long it_beg = total * wk / G, it_end = total * (wk + 1) / G;
     const int my_iters = (int)(it_end - it_beg);
     const int prefill = my_iters < p.stages ? my_iters : p.stages;    // weight stages requested during set-up
+    // work unit -> this CTA's 128-row tile, and the row coordinate of that tile in the weight map
+    auto tile_of = [&](int wt) { return PAIR ? 2 * wt + rank : wt; };
+    auto w_row = [&](int wt) { return p.swiglu_f ? tile_of(wt) * 64 : tile_of(wt) * TILE_M; };
+    // barrier (in the even CTA when PAIR) that counts the bytes of ring stage s
+    auto full_bar = [&](int s) { return PAIR ? mapa_shared(smem_u32(&sm->full[s]), 0) : smem_u32(&sm->full[s]); };
+    auto load_w = [&](uint32_t dst, int wt, int kc, uint32_t bar, uint64_t pol) {
+        if constexpr (PAIR) tma_load_4d_pair(dst, &tm_w, 0, w_row(wt), 0, kc * p.ks, bar, pol);
+        else tma_load_4d(dst, &tm_w, 0, w_row(wt), 0, kc * p.ks, bar, pol);
+    };
+    auto load_x = [&](uint32_t dst, int kc, uint32_t bar, uint64_t pol) {
+        if constexpr (PAIR) tma_load_4d_pair(dst, &tm_x, 0, rank * nb_cta, 0, kc * p.ks, bar, pol);
+        else tma_load_4d(dst, &tm_x, 0, 0, 0, kc * p.ks, bar, pol);
+    };
+    const uint32_t full_tx = PAIR ? 2 * stage_bytes : stage_bytes;      // both CTAs' loads land on the even CTA's barrier
 
     // accumulator buffers are EPI_CHUNK-aligned so that a 32-column read never leaves the allocation
     const uint32_t buf_cols = (uint32_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK);
@@ -68,33 +92,41 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
     }
+    // Weights never change, so the first ring-full of weight stages is requested during set-up: their latency
+    // overlaps the tensor-memory allocation, the CTA barrier and the tail of the preceding kernel; the activations
+    // of those stages follow after the dependency wait.
+    auto prefill_weights = [&] {
+        uint64_t pol_first;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+        int wt = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)wt * p.kiters);
+        for (int i = 0; i < prefill; ++i) {
+            if (rank == 0) mbar_expect_tx(smem_u32(&sm->full[i]), full_tx);
+            load_w(tiles_addr + i * stage_bytes, wt, kc, full_bar(i), pol_first);
+            if (++kc == p.kiters) { kc = 0; ++wt; }
+        }
+    };
     if (threadIdx.x == 0) {
+        const uint32_t epi_warps = TWO ? 8 : 4;
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&sm->full[s]), 1); mbar_init(smem_u32(&sm->empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), TWO ? 8 : 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sm->tmem_full[b]), 1); mbar_init(smem_u32(&sm->tmem_empty[b]), PAIR ? 2 * epi_warps : epi_warps); }
         mbar_init(smem_u32(&sm->drain), 1);
         sm->abort_flag = 0;
         sm->last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // This thread is also the TMA producer.  Weights never change, so the first ring-full of weight
-        // stages is requested right here: their latency overlaps the rest of the set-up (tensor-memory
-        // allocation, CTA barrier) and the tail of the preceding kernel; the activations of those stages
-        // follow after the dependency wait.
-        uint64_t pol_first;
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
-        int tile = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)tile * p.kiters);
-        for (int i = 0; i < prefill; ++i) {
-            const uint32_t full = smem_u32(&sm->full[i]);
-            mbar_expect_tx(full, stage_bytes);
-            tma_load_4d(tiles_addr + i * stage_bytes, &tm_w, 0, p.swiglu_f ? tile * 64 : tile * TILE_M, 0, kc * p.ks, full, pol_first);
-            if (++kc == p.kiters) { kc = 0; ++tile; }
-        }
+        if constexpr (!PAIR) prefill_weights();            // this thread is also the TMA producer
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (PAIR) {       // the same warp of both CTAs: columns are reserved in both tensor memories
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
-    __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();     // the other CTA's barriers exist before anything is counted on them
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
@@ -103,20 +135,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
+            if constexpr (PAIR) prefill_weights();
             uint64_t pol_stream, pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            // (tile, kc) advance incrementally: a 64-bit division per stage would cost this single thread
+            // (work unit, kc) advance incrementally: a 64-bit division per stage would cost this single thread
             // more cycles than the loads it issues
-            int tile = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)tile * p.kiters);
+            int wt = (int)(it_beg / p.kiters), kc = (int)(it_beg - (long long)wt * p.kiters);
             if (prefill > 0) {
                 pdl_wait();                                    // the activations belong to the preceding kernel until now
                 for (int q = 0; q < prefill; ++q) {            // activations of the stages whose weights went out during set-up
-                    tma_load_4d(tiles_addr + q * stage_bytes + a_bytes, &tm_x, 0, 0, 0, kc * p.ks, smem_u32(&sm->full[q]), pol_keep);
-                    if (++kc == p.kiters) { kc = 0; ++tile; }
+                    load_x(tiles_addr + q * stage_bytes + a_bytes, kc, full_bar(q), pol_keep);
+                    if (++kc == p.kiters) { kc = 0; ++wt; }
                 }
                 issued = prefill;
                 if (prefill == p.stages) phase = 1; else stage = (uint32_t)prefill;
@@ -124,34 +157,39 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             for (int i = prefill; i < my_iters && ok; ++i) {
                 ok = mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_TMA);
                 if (!ok) break;
-                const uint32_t full = smem_u32(&sm->full[stage]);
+                const uint32_t full = full_bar(stage);
                 const uint32_t a_dst = tiles_addr + stage * stage_bytes, b_dst = a_dst + a_bytes;
-                mbar_expect_tx(full, stage_bytes);
-                tma_load_4d(a_dst, &tm_w, 0, p.swiglu_f ? tile * 64 : tile * TILE_M, 0, kc * p.ks, full, pol_stream);
-                tma_load_4d(b_dst, &tm_x, 0, 0, 0, kc * p.ks, full, pol_keep);
+                if (rank == 0) mbar_expect_tx(smem_u32(&sm->full[stage]), full_tx);
+                load_w(a_dst, wt, kc, full, pol_stream);
+                load_x(b_dst, kc, full, pol_keep);
                 ++issued;
                 if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
-                if (++kc == p.kiters) { kc = 0; ++tile; }
+                if (++kc == p.kiters) { kc = 0; ++wt; }
             }
             if (!ok) {
-                // drain: wait (bounded) until every load issued into the ring has landed
+                // drain: wait (bounded) until every load issued into the ring has landed (the even CTA sees the
+                // pair's byte counts; the odd one relies on the cluster barrier at the end of the kernel)
                 const int inflight = issued < p.stages ? issued : p.stages;
                 uint32_t s = stage, ph = phase;
-                for (int q = 0; q < inflight; ++q) {
+                for (int q = 0; q < inflight && rank == 0; ++q) {
                     if (s == 0) { s = p.stages - 1; ph ^= 1; } else --s;
                     for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->full[s]), ph); ++spin) __nanosleep(64);
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_f16(p.nb);
+        // ------------------------------------------------ MMA issuer (PAIR: in the even CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_f16(p.nb, false, PAIR ? 256 : 128);
             uint32_t stage = 0, phase = 0, buf = 0, buf_phase = 0;
             long long units = 0;
             bool ok = true;
             long long it = it_beg;
-            int tile = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)tile * p.kiters);   // later units: next tile, k0 = 0
+            int k0 = (int)(it_beg - (it_beg / p.kiters) * p.kiters);   // later units: next work unit, k0 = 0
+            auto commit = [&](uint64_t* bar) {                 // PAIR: the barrier at this offset in both CTAs
+                if constexpr (PAIR) tc_commit_pair_both(smem_u32(bar));
+                else tc_commit(smem_u32(bar));
+            };
             while (it < it_end && ok) {
                 const long long left = it_end - it;
                 const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
@@ -168,23 +206,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     for (int sl = 0; sl < nslab; ++sl) {
                         const uint64_t adesc = smem_desc_sw128(a_addr + sl * a_slab), bdesc = smem_desc_sw128(b_addr + sl * b_slab);
 #pragma unroll
-                        for (int j = 0; j < TILE_K / UMMA_K; ++j)   // +32 bytes along k inside the swizzle row per step
-                            tc_mma_f16(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, (kc > k0 || sl > 0 || j > 0) ? 1u : 0u);
+                        for (int j = 0; j < TILE_K / UMMA_K; ++j) {   // +32 bytes along k inside the swizzle row per step
+                            const uint32_t acc = (kc > k0 || sl > 0 || j > 0) ? 1u : 0u;
+                            if constexpr (PAIR) tc_mma_f16_pair(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, acc);
+                            else tc_mma_f16(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, acc);
+                        }
                     }
-                    tc_commit(smem_u32(&sm->empty[stage]));    // stage is free once these MMAs have read it
+                    commit(&sm->empty[stage]);                 // stage is free once these MMAs have read it
                     if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&sm->tmem_full[buf]));       // accumulator complete
+                commit(&sm->tmem_full[buf]);                    // accumulator complete
                 ++units;
                 if (++buf == 2) { buf = 0; buf_phase ^= 1; }
                 it += (k1 - k0);
-                ++tile;
                 k0 = 0;
             }
             if (!ok) {
                 // make sure no MMA is still running before TMEM goes away
-                tc_commit(smem_u32(&sm->drain));
+                if constexpr (PAIR) tc_commit_pair_local(smem_u32(&sm->drain));
+                else tc_commit(smem_u32(&sm->drain));
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain), 0); ++spin) __nanosleep(64);
             }
         }
@@ -198,16 +239,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         auto fused = [&](int tile_, int c0_, float (&v_)[32]) { epilogue_chunk<GROUPS>(p, sm, grp, tile_, row, c0_, v_); };
         const int et = threadIdx.x - 64;                       // 0..255 among epilogue threads
         const size_t slot_elems = (size_t)buf_cols * TILE_M;   // columns padded to whole 32-wide chunks
+        // partial-tile buffer of worker c's CTA that works on the same tile parity as this one
+        auto part_of = [&](int c) { return p.part + (size_t)(PAIR ? 2 * c + rank : c) * 2 * slot_elems; };
+        // the accumulator buffer is free again: counted on the MMA issuer's barrier
+        const uint32_t tmem_empty0 = PAIR ? mapa_shared(smem_u32(&sm->tmem_empty[0]), 0) : smem_u32(&sm->tmem_empty[0]);
+        auto release_acc = [&](uint32_t b) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_cluster(tmem_empty0 + b * (uint32_t)sizeof(uint64_t));
+                else mbar_arrive(tmem_empty0 + b * (uint32_t)sizeof(uint64_t));
+            }
+        };
         // Epilogue of a complete tile.  split = false: the accumulator holds the whole sum.  split = true: this CTA
         // (the tile's first contributor) has its share in tensor memory and adds the other contributors' partial
-        // tiles from the workspace in CTA order (fixed order -> reproducible); each one's 32 loads go out together.
+        // tiles from the workspace in worker order (fixed order -> reproducible); each one's 32 loads go out together.
         auto finish_tile = [&](int tile_, uint32_t t_addr_, bool split, int c_first_, int c_last_) {
             for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += GROUPS * EPI_CHUNK) {
                 float v[32];
                 tc_ld32(t_addr_ + c0, v);                  // may run past nb, never past the buffer
                 if (split) {
                     for (int c = c_first_ + 1; c <= c_last_; ++c) {      // later contributors always use their slot 0
-                        const float* src = p.part + (size_t)c * 2 * slot_elems + (size_t)c0 * TILE_M + row;
+                        const float* src = part_of(c) + (size_t)c0 * TILE_M + row;
                         float t[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * TILE_M);
@@ -239,8 +292,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
         long long it = it_beg;
-        int tile = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)tile * p.kiters);
-        for (; it < it_end && ok; ++tile, k0 = 0) {
+        int wt = (int)(it_beg / p.kiters), k0 = (int)(it_beg - (long long)wt * p.kiters);
+        for (; it < it_end && ok; ++wt, k0 = 0) {
+            const int tile = tile_of(wt);
             const long long left = it_end - it;
             const int k1 = (p.kiters - k0 < left) ? p.kiters : (int)(k0 + left);
             const bool whole = (k0 == 0 && k1 == p.kiters) && p.epi.mode != EPI_DEFER;
@@ -250,18 +304,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
-            // A tile some CTAs share is finished by its FIRST contributor: for that CTA the tile is the last unit of
+            // A tile some workers share is finished by its FIRST contributor: for that CTA the tile is the last unit of
             // its range, so it gets here last in time, while every other contributor handles its share as the first
             // unit of its range (or as its only one), stores it and counts itself in without ever waiting.  The
             // finisher keeps its own share in tensor memory and waits (bounded) for the others; they run at the same
             // time on other SMs and depend on nobody, so the wait is short: the store and count of a contributor
             // that ended together with the finisher.
-            const int c_first = p.tile_first[tile], c_last = c_first + p.tile_count[tile] - 1;
+            const int c_first = p.tile_first[wt], c_last = c_first + p.tile_count[wt] - 1;
             bool finish = whole;
             if (!whole && p.epi.mode != EPI_DEFER) {
                 if (et == 0) {
                     int fl = 0;
-                    if (cta == c_first) {
+                    if (wk == c_first) {
                         fl = 1;
                         uint32_t spin = 0;
                         while (ld_acquire_gpu(p.counters + tile) != c_last - c_first) {
@@ -290,9 +344,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                     for (int j = 0; j < 32; ++j) __stcg(mine + (size_t)(c0 + j) * TILE_M + row, v[j]);
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty[buf]));
+            release_acc(buf);
             if (!finish && p.epi.mode != EPI_DEFER) {
                 // count this arrival: the barrier orders every thread's stores before thread 0's
                 // release, and the release is cumulative over them
@@ -305,40 +357,70 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     }
 
     tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    if constexpr (PAIR) {
+        // neither CTA may leave while the other's MMAs can still read its shared memory or write its tensor memory
+        if (warp == 0 && lane == 0 && rank != 0 && *abort_flag)
+            for (int q = 0; q < 64; ++q) __nanosleep(1000);      // gave up: let this CTA's loads in flight land
+        cluster_sync_all();
+        if (warp == 1) {
+            tc_fence_after();
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+        }
+    } else {
+        __syncthreads();
+        if (warp == 1) {
+            tc_fence_after();
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+        }
     }
 }
 
 // ---------------------------------------------------------------- host side
-size_t smem_bytes_for(int nb, int ks, int stages) {
-    return 1024 + (size_t)stages * ks * (TILE_M * TILE_K * 2 + (size_t)nb * TILE_K * 2) + sizeof(Smem);
+size_t smem_bytes_for(int nb_cta, int ks, int stages) {      // nb_cta: activation rows one CTA loads per k-slab
+    return 1024 + (size_t)stages * ks * (TILE_M * TILE_K * 2 + (size_t)nb_cta * TILE_K * 2) + sizeof(Smem);
 }
 
-int pick_stages(int nb, int ks) {
+int pick_stages(int nb_cta, int ks) {
     int s = MAX_STAGES;
-    while (s > 2 && smem_bytes_for(nb, ks, s) > 227 * 1024) --s;
+    while (s > 2 && smem_bytes_for(nb_cta, ks, s) > 227 * 1024) --s;
     return s;
+}
+
+int tiles_of(int m, int epi_mode) { return (epi_mode == EPI_SWIGLU) ? (m / 2) / 64 : (m + TILE_M - 1) / TILE_M; }
+
+// CTA pairs (one activation half per CTA) pay off once the activation slab outweighs the weight tile.
+bool use_pairs(const ghd_ctx* c, int n, int m, int epi_mode) {
+    const int nb = ((n + 15) / 16) * 16;
+    const int tiles = tiles_of(m, epi_mode);
+    if (c->opt_gemm_pair == 1 || tiles % 2 || tiles < 2 || nb < 32 || c->sm_count < 2) return false;
+    return c->opt_gemm_pair == 2 || nb > 128;
+}
+
+// CTAs of a launch before the clamp to the work there is
+int base_ctas(const ghd_ctx* c, bool pair) {
+    int ctas = c->opt_gemm_ctas > 0 && c->opt_gemm_ctas < c->sm_count ? c->opt_gemm_ctas : c->sm_count;
+    if (pair) ctas &= ~1;
+    return ctas < (pair ? 2 : 1) ? (pair ? 2 : 1) : ctas;
 }
 
 }  // namespace
 
 bool gemm_tc_supported(const ghd_ctx* c, int n, int k, int m, int epi_mode) {
     if (c->cfg.dtype != GHD_F16 || n < 1 || n > GHD_MAX_NODES || k % TILE_K || k < TILE_K) return false;
-    const int n_tiles = (epi_mode == EPI_SWIGLU) ? (m / 2) / 64 : (m + TILE_M - 1) / TILE_M;
+    const int n_tiles = tiles_of(m, epi_mode);
     if (n_tiles < 1 || n_tiles > MAX_TILES) return false;
     if (epi_mode == EPI_SWIGLU && (m / 2) % 64) return false;
     if (epi_mode == EPI_ROPE_KV && ((m / 3) % TILE_M || m % 3)) return false;
     if (epi_mode == EPI_RESID_NORM && (m % TILE_M || m / TILE_M > SSQ_MAX_TILES)) return false;
     if (epi_mode == EPI_DEFER) {
-        int ctas = c->opt_gemm_ctas > 0 && c->opt_gemm_ctas < c->sm_count ? c->opt_gemm_ctas : c->sm_count;
-        const int ks = (((n + 15) / 16) * 16 <= 128) ? 2 : 1;
+        const bool pair = use_pairs(c, n, m, epi_mode);
+        int workers = base_ctas(c, pair) / (pair ? 2 : 1);
+        const int nb = ((n + 15) / 16) * 16;
+        const int ks = c->opt_gemm_burst > 0 ? (c->opt_gemm_burst > 4 ? 4 : c->opt_gemm_burst) : ((pair ? nb / 2 : nb) <= 128 ? 2 : 1);
         const int kch = (k / TILE_K + ks - 1) / ks;
-        const long long total = (long long)n_tiles * kch;
-        if (ctas > total) ctas = (int)total;
-        if (m % 4 || m > 16384 || total / ctas + 1 > kch || total / ctas < 1) return false;
+        const long long total = (long long)(n_tiles / (pair ? 2 : 1)) * kch;
+        if (workers > total) workers = (int)total;
+        if (m % 4 || m > 16384 || total / workers + 1 > kch || total / workers < 1) return false;
     }
     return true;
 }
@@ -355,52 +437,57 @@ ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, 
     p.k = k;
     p.m = m;
     p.swiglu_f = (epi.mode == EPI_SWIGLU) ? m / 2 : 0;
-    p.n_tiles = p.swiglu_f ? p.swiglu_f / 64 : (m + TILE_M - 1) / TILE_M;
-    p.ks = c->opt_gemm_burst > 0 ? c->opt_gemm_burst : (p.nb <= 128 ? 2 : 1);
+    p.n_tiles = tiles_of(m, epi.mode);
+    p.pair = use_pairs(c, n, m, epi.mode) ? 1 : 0;
+    p.n_work = p.pair ? p.n_tiles / 2 : p.n_tiles;
+    const int nb_cta = p.pair ? p.nb / 2 : p.nb;
+    p.ks = c->opt_gemm_burst > 0 ? c->opt_gemm_burst : (nb_cta <= 128 ? 2 : 1);
     if (p.ks > 4) p.ks = 4;
     p.kslabs = k / TILE_K;
     p.kiters = (p.kslabs + p.ks - 1) / p.ks;
-    p.stages = pick_stages(p.nb, p.ks);
+    p.stages = pick_stages(nb_cta, p.ks);
     if (c->opt_gemm_stages >= 2 && c->opt_gemm_stages < p.stages) p.stages = c->opt_gemm_stages;
     p.part = c->gemm_part;
     p.counters = c->counters;
     p.status = c->status;
     p.epi = epi;
     if (!tmap_slabs(c, w, (uint64_t)m, (uint64_t)k, p.swiglu_f ? 2 : 1, p.swiglu_f ? 64 : TILE_M, (uint32_t)p.ks, &plan->tm_w) ||
-        !tmap_slabs(c, x, (uint64_t)n, (uint64_t)k, 1, (uint32_t)p.nb, (uint32_t)p.ks, &plan->tm_x)) {
+        !tmap_slabs(c, x, (uint64_t)n, (uint64_t)k, 1, (uint32_t)nb_cta, (uint32_t)p.ks, &plan->tm_x)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: tensor map encoding failed");
         return GHD_ECUDA;
     }
-    const long long total = (long long)p.n_tiles * p.kiters;
-    int ctas = c->opt_gemm_ctas > 0 ? c->opt_gemm_ctas : c->sm_count;
-    if (ctas > c->sm_count) ctas = c->sm_count;
-    if (c->opt_gemm_ctas <= 0 && epi.mode != EPI_DEFER && p.n_tiles < c->sm_count) {
-        // Fewer tiles than SMs: every CTA range is shorter than a tile.  With n_tiles * q / (q - 1) CTAs each
-        // range is (q-1)/q of a tile and always touches a tile boundary, so no tile is shared by three CTAs
-        // and no CTA's only unit sits strictly inside a tile (those finish together and take the slow
+    // workers: CTAs, or clusters of two CTAs; they share the flattened (work unit, k-chunk) space
+    const int per = p.pair ? 2 : 1;
+    const long long total = (long long)p.n_work * p.kiters;
+    int workers = base_ctas(c, p.pair != 0) / per;
+    if (c->opt_gemm_ctas <= 0 && epi.mode != EPI_DEFER && p.n_work < workers) {
+        // Fewer work units than workers: every range is shorter than a unit.  With n_work * q / (q - 1) workers each
+        // range is (q-1)/q of a unit and always touches a unit boundary, so no tile is shared by three workers
+        // and no worker's only share sits strictly inside a tile (those finish together and take the slow
         // split-tile path).  Take the largest such count that fits the SMs.
         int best = 0;
         for (int q = 2; q <= 64; ++q)
-            if ((p.n_tiles * q) % (q - 1) == 0) {
-                const int g = p.n_tiles * q / (q - 1);
-                if (g <= c->sm_count && g > best) best = g;
+            if ((p.n_work * q) % (q - 1) == 0) {
+                const int g = p.n_work * q / (q - 1);
+                if (g <= workers && g > best) best = g;
             }
-        if (best >= c->sm_count * 3 / 4) ctas = best;
+        if (best >= workers * 3 / 4) workers = best;
     }
-    if (ctas > total) ctas = (int)total;
+    if (workers > total) workers = (int)total;
+    const int ctas = workers * per;
     p.ctas = ctas;
-    plan->smem = smem_bytes_for(p.nb, p.ks, p.stages);
-    for (int t = 0; t < p.n_tiles; ++t) {
+    plan->smem = smem_bytes_for(nb_cta, p.ks, p.stages);
+    for (int t = 0; t < p.n_work; ++t) {
         const long long t_first = (long long)t * p.kiters;
-        const int c_first = (int)(((t_first + 1) * ctas + total - 1) / total) - 1;
-        const int c_last = (int)(((t_first + p.kiters) * ctas + total - 1) / total) - 1;
+        const int c_first = (int)(((t_first + 1) * workers + total - 1) / total) - 1;
+        const int c_last = (int)(((t_first + p.kiters) * workers + total - 1) / total) - 1;
         p.tile_first[t] = (unsigned short)c_first;
         p.tile_count[t] = (unsigned char)(c_last - c_first + 1);
-        p.tile_slot[t] = (total * c_first / ctas >= t_first) ? 0 : 1;
+        p.tile_slot[t] = (total * c_first / workers >= t_first) ? 0 : 1;
     }
     plan->pending.active = 0;
     if (epi.mode == EPI_DEFER) {
-        if (total / ctas + 1 > p.kiters) {                // a CTA range must touch at most two tiles
+        if (total / workers + 1 > p.kiters) {             // a worker's range must touch at most two work units
             snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: deferred reduction needs n_tiles <= CTAs");
             return GHD_EUNSUPPORTED;
         }
@@ -411,10 +498,12 @@ ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, 
         pp.total = total;
         pp.slot_elems = (size_t)((p.nb + EPI_CHUNK - 1) / EPI_CHUNK * EPI_CHUNK) * TILE_M;
         pp.m = m;
+        pp.stride = per;                                  // CTA pairs: a tile's contributors are every other CTA
         for (int t = 0; t < p.n_tiles && t < 128; ++t) {
-            pp.first_cta[t] = p.tile_first[t];
-            pp.n_contrib[t] = p.tile_count[t];
-            pp.first_slot[t] = p.tile_slot[t];
+            const int wt = t / per;
+            pp.first_cta[t] = (unsigned short)(p.tile_first[wt] * per + t % per);
+            pp.n_contrib[t] = p.tile_count[wt];
+            pp.first_slot[t] = p.tile_slot[wt];
         }
     }
     return GHD_OK;
@@ -425,8 +514,10 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     const ghd_status s = plan_gemm_tc(c, x, w, n, k, m, epi, &plan);
     if (s != GHD_OK) return s;
     if (!c->attr_gemm) {       // per context: the attribute belongs to the device the context was created on
-        if (cudaFuncSetAttribute(k_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(k_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+        if (cudaFuncSetAttribute(k_gemm_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gemm_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gemm_tc<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gemm_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: cannot raise dynamic shared memory: %s", cudaGetErrorString(cudaGetLastError()));
             return GHD_ECUDA;
         }
@@ -434,8 +525,15 @@ ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k
     }
     if (plan.pending.active) c->pending = plan.pending;
     const bool two = c->opt_gemm_epi ? c->opt_gemm_epi == 2 : plan.p.nb > EPI_CHUNK;
-    if (two) launch_k(c, true, k_gemm_tc<true>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
-    else launch_k(c, true, k_gemm_tc<false>, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    if (plan.p.pair) {
+        c->path_count[GHD_PATH_GEMM_PAIR]++;
+        if (two) launch_kc(c, true, 2, k_gemm_tc<true, true>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+        else launch_kc(c, true, 2, k_gemm_tc<false, true>, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    } else if (two) {
+        launch_k(c, true, k_gemm_tc<true, false>, plan.p.ctas, THREADS_TC, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    } else {
+        launch_k(c, true, k_gemm_tc<false, false>, plan.p.ctas, THREADS, plan.smem, plan.tm_w, plan.tm_x, plan.p);
+    }
     return GHD_OK;
 }
 

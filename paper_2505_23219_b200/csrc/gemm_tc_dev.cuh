@@ -20,15 +20,16 @@ constexpr int MAX_TILES = 256;
 struct GemmParams {
     int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
     int n_tiles, kiters, stages;     // kiters = k-chunks per tile; a chunk = ks column slabs of 64 = one pipeline stage
+    int n_work, pair;                // work units dealt to the workers: tiles (one CTA each), or tile pairs (pair = 1: one cluster of two CTAs each)
     int ks, kslabs;                  // slabs per stage, slabs per weight row (k / 64)
     int swiglu_f;                    // d_ffn when the tile is [64 gate rows | 64 up rows], else 0
-    int ctas;                        // CTAs that share the flattened (tile, k-chunk) space
+    int ctas;                        // CTAs of the launch; ctas / (1 + pair) workers share the flattened (work unit, k-chunk) space
     float* part;                     // [ctas][2][nb][128] float partial tiles
     int* counters;                   // [n_tiles] arrival counters, zero on entry and on exit
     int* status;
     EpiArgs epi;
-    // per tile, worked out on the host (64-bit divisions are slow on the device): first contributing
-    // CTA, number of contributors, slot of the first contributor (the others use slot 0)
+    // per work unit, worked out on the host (64-bit divisions are slow on the device): first contributing
+    // worker, number of contributors, slot of the first contributor (the others use slot 0)
     unsigned short tile_first[MAX_TILES];
     unsigned char tile_count[MAX_TILES], tile_slot[MAX_TILES];
 };

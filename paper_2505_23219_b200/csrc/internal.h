@@ -65,6 +65,7 @@ struct StepGraph;
 // slot 0, its second (if any) in slot 1, each slot [columns][128 rows] float.
 struct PendingPartials {
     int active, kiters, ctas, m;
+    int stride;       // CTA distance between two contributors of a tile (2 when CTA pairs ran the projection)
     long long total;
     size_t slot_elems;
     // per 128-row tile, worked out on the host (integer divisions are expensive on the device):
@@ -82,7 +83,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm, opt_gemm_pair;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;

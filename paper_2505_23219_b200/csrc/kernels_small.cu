@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(1024) k_fold_pending(float* __restrict__ xres,
                     t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (cb + q < cnt) {
                         const int slot = (cb + q == 0) ? slot0 : 0;
-                        t[q] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(c_first + cb + q) * 2 + slot) * pp.slot_elems +
+                        t[q] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(c_first + (cb + q) * pp.stride) * 2 + slot) * pp.slot_elems +
                                                                       (size_t)node * 128 + row));
                     }
                 }

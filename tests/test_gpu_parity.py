@@ -176,6 +176,41 @@ def test_linear_tcgen05_path(ghd, n, k, m):
         assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
 
 
+PAIR_SHAPES = [(17, 320, 130), (33, 512, 256), (64, 4096, 1024), (100, 1024, 1001), (128, 512, 768), (200, 2048, 256),
+               (256, 1024, 512), (256, 4096, 2048)]
+
+
+@pytest.mark.parametrize("n,k,m", PAIR_SHAPES)
+def test_linear_tcgen05_on_cta_pairs(ghd, n, k, m):
+    """Clusters of two CTAs (cta_group::2): each CTA loads its weight tile and half of the activation rows."""
+    ctx = make_ctx(ghd, SMALL16, 128, 256)
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PATH, 2)
+    ghd.ghd_set_option(ctx, ghd.OPT_GEMM_PAIR, 2)
+    x = wl.normal((n, k), 331, 1.0, dtype="f16")
+    w = wl.normal((m, k), 332, 0.02, dtype="f16")
+    xd, wd = to_dev(x), to_dev(w)
+    y = ghd.ghd_linear(ctx, xd, wd)
+    ghd.ghd_sync_status(ctx)
+    assert ghd.ghd_path_count(ctx, ghd.PATH_GEMM_PAIR) == 1, "the paired kernel did not run"
+    want = oracle.linear(x, w)
+    assert max_rel_err(y.cpu().numpy(), want) <= 2e-5
+    y2 = ghd.ghd_linear(ctx, xd, wd)
+    ghd.ghd_sync_status(ctx)
+    assert np.array_equal(y.cpu().numpy(), y2.cpu().numpy())  # fixed reduction order -> reproducible
+    for ctas in (2, 6, 64):                                   # result must not depend on the work split
+        ghd.ghd_set_option(ctx, ghd.OPT_GEMM_CTAS, ctas)
+        y3 = ghd.ghd_linear(ctx, xd, wd)
+        ghd.ghd_sync_status(ctx)
+        assert max_rel_err(y3.cpu().numpy(), want) <= 2e-5
+
+
+@pytest.mark.parametrize("n,L", [(13, 100), (64, 77), (100, 300), (128, 9), (200, 5), (256, 31)])
+def test_small_layers_with_projections_on_cta_pairs(ghd, n, L):
+    import paper_2505_23219_b200 as g
+    ctx = _layer_case(ghd, SMALL16_DH128, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6), opts=[(g.OPT_GEMM_PAIR, 2)])
+    assert ghd.ghd_path_count(ctx, ghd.PATH_GEMM_PAIR) >= (3 if n > 16 else 0)     # QKV, O, down (gate/up has 11 tiles)
+
+
 def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0, on_device=False):
     Lmax = L + n + (150 if on_device else 3)               # on_device: the kernels see cache rows far past kv_len + n
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
