@@ -289,6 +289,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             }
             epi_all();
         }
+        // Projections into the residual stream finish their split tiles in SLICES: every contributor stores its share
+        // and counts itself in; when its range is done it waits (bounded) until all contributors of the tile have
+        // arrived and finishes its own share of the tile's node columns (sum of the partial tiles in worker order,
+        // residual add, gain-weighted copy, sums of squares).  All SMs take part in the reduction, nobody keeps an
+        // accumulator waiting, and the epilogue needs no exchange between rows.
+        const bool sliced = p.epi.mode == EPI_RESID_NORM || p.epi.mode == EPI_RESID;
+        int pend_wt[2], n_pend = 0;
         uint32_t buf = 0, buf_phase = 0;
         bool ok = true;
         long long it = it_beg;
@@ -312,7 +319,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             // that ended together with the finisher.
             const int c_first = p.tile_first[wt], c_last = c_first + p.tile_count[wt] - 1;
             bool finish = whole;
-            if (!whole && p.epi.mode != EPI_DEFER) {
+            if (!whole && sliced) pend_wt[n_pend++] = wt;
+            if (!whole && p.epi.mode != EPI_DEFER && !sliced) {
                 if (et == 0) {
                     int fl = 0;
                     if (wk == c_first) {
@@ -353,6 +361,77 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             }
             if (++buf == 2) { buf = 0; buf_phase ^= 1; }
             it += (k1 - k0);
+        }
+        for (int q = 0; q < n_pend && ok; ++q) {
+            const int swt = pend_wt[q], tile = tile_of(swt);
+            const int c_first = p.tile_first[swt], cnt = p.tile_count[swt], idx = wk - c_first;
+            if (et == 0) {
+                uint32_t spin = 0;
+                while (ld_acquire_gpu(p.counters + tile) != cnt) {
+                    if (++spin >= SPIN_LIMIT) { *abort_flag = 1; atomicCAS(p.status, DEV_OK, DEV_TIMEOUT_GRID); break; }
+                    __nanosleep(spin > 64 ? 64 : 20);
+                }
+            }
+            epi_all();
+            ok = (*abort_flag == 0);
+            if (!ok) break;
+            constexpr int CB = 8, P = TWO ? 2 : 1;             // columns per batch of a thread; column phases
+            const int lo = p.n * idx / cnt, hi = p.n * (idx + 1) / cnt;
+            const int phase = et >> 7;                          // row = et & 127 (the thread's feature), quad = its warp
+            const int f = tile * TILE_M + row;
+            const unsigned m = (unsigned)p.m;
+            const bool norm = p.epi.mode == EPI_RESID_NORM;
+            const float g = (norm && f < p.m) ? __half2float(__ldg((const __half*)p.epi.gain + f)) : 0.f;
+            const int slot0 = p.tile_slot[swt];
+            for (int j0 = lo + phase; j0 < hi; j0 += P * CB) {
+                float acc[CB], old[CB];
+#pragma unroll
+                for (int b = 0; b < CB; ++b) {
+                    const int col = j0 + b * P;
+                    acc[b] = 0.f;
+                    old[b] = (col < hi && f < p.m) ? __ldcg(p.epi.out_f32 + (size_t)col * m + f) : 0.f;
+                }
+                for (int c = 0; c < cnt; c += 4) {               // four contributors' loads in flight together
+                    float t[4][CB];
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const float* src = part_of(c_first + c + cc) + (size_t)((c + cc == 0) ? slot0 : 0) * slot_elems + row;
+#pragma unroll
+                        for (int b = 0; b < CB; ++b) {
+                            const int col = j0 + b * P;
+                            t[cc][b] = (c + cc < cnt && col < hi) ? __ldcg(src + (size_t)col * TILE_M) : 0.f;
+                        }
+                    }
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                        for (int b = 0; b < CB; ++b) acc[b] += t[cc][b];
+                }
+#pragma unroll
+                for (int b = 0; b < CB; ++b) {
+                    const int col = j0 + b * P;
+                    const float v = acc[b] + old[b];
+                    if (col < hi && f < p.m) {
+                        p.epi.out_f32[(size_t)col * m + f] = v;
+                        if (norm) ((__half*)p.epi.xg_out)[(size_t)col * m + f] = __float2half_rn(v * g);
+                    }
+                    if (norm) {
+                        float sq = (col < hi && f < p.m) ? v * v : 0.f;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                        if (lane == 0 && col < hi) sm->ssq_slice[quad][col - lo] = sq;
+                    }
+                }
+            }
+            epi_all();
+            if (norm && et < hi - lo)
+                p.epi.ssq_out[(size_t)tile * SSQ_PITCH + lo + et] =
+                    (sm->ssq_slice[0][et] + sm->ssq_slice[1][et]) + (sm->ssq_slice[2][et] + sm->ssq_slice[3][et]);
+            epi_all();
+            if (et == 0 && atom_add_acq_rel_gpu(p.counters + DONE_OFF + tile, 1) == cnt - 1) {
+                p.counters[tile] = 0;                           // everybody has passed the wait: ready for the next launch
+                p.counters[DONE_OFF + tile] = 0;
+            }
         }
     }
 

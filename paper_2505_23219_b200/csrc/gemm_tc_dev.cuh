@@ -16,6 +16,7 @@ constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
 constexpr int THREADS = 192;
 constexpr int THREADS_TC = 320;      // k_gemm_tc: producer warp, MMA warp, two groups of four epilogue warps
 constexpr int MAX_TILES = 256;
+constexpr int DONE_OFF = 2048;       // counters[DONE_OFF + tile]: contributors that have finished their slice of a split tile
 
 struct GemmParams {
     int n, nb, k, m;                 // nodes, padded nodes (MMA N), reduction length, output features
@@ -48,6 +49,7 @@ struct Smem {
     float stage_x[EPI_CHUNK][TILE_M + 1];   // epilogue exchange buffer (rotary pairs, gate/up pairs)
     float colscale[GHD_MAX_NODES];          // 1 / rms of every input row (projections that read un-normalised rows)
     float ssq_part[2][4][32];               // per epilogue group and warp: sums of squares of 32 rows x 32 nodes
+    float ssq_slice[4][GHD_MAX_NODES / 2];  // slice finishing: per 32-row warp, sums of squares of the slice's columns
 };
 
 // s[j] (j < 32) summed over the 32 lanes of the warp; lane L returns the total of column L.
