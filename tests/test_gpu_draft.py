@@ -226,3 +226,75 @@ def test_self_drafting_loop_with_the_cache_length_on_the_device(ghd, shape, grap
     for (ok, ov), kv in zip(o_caches, gkv):
         assert max_rel_err(kv.k.float().cpu().numpy()[:, L0:L0 + keep], ok[:, L0:L0 + keep]) <= tol
         assert max_rel_err(kv.v.float().cpu().numpy()[:, L0:L0 + keep], ov[:, L0:L0 + keep]) <= tol
+
+
+def test_self_drafting_steps_captured_in_one_cuda_graph(ghd):
+    """S consecutive draft / verify / accept / commit steps recorded ONCE into a CUDA graph by the caller and replayed:
+    possible because nothing between the steps needs the host (cache length, accepted path, next root and next drafts
+    all stay on the device)."""
+    import torch
+    shape = SMALL16
+    L0, steps, width = 12, 6, 14
+    acc = [[0.6, 0.3, 0.2, 0.1], [0.5, 0.3, 0.1], [0.4, 0.2]]
+    most = steps * (len(acc) + 1)
+    Lmax = L0 + most + width + 1
+    head = wl.head_weights(shape, 46)
+    layers = [wl.layer_weights(shape, 46, l, random_gains=True) for l in range(shape.n_layers)]
+    fresh = lambda: [wl.kv_cache(shape, 46, l, L0, Lmax) for l in range(shape.n_layers)]
+    o_caches = fresh()
+    g, gaps, first_logits = [5], [], None
+    for s in range(most + 1):
+        vis, _, pos = oracle.tree_build([-1], L0 + s)
+        logits, am = oracle.step(shape, head, layers, o_caches, L0 + s, vis, pos, [g[-1]])
+        first_logits = logits[0].copy() if first_logits is None else first_logits
+        top = np.partition(logits[0], -2)
+        gaps.append(float(top[-1] - top[-2]))
+        g.append(int(am[0]))
+    topk = tuple(len(a) for a in acc)
+    parent, paths, _ = arca.build_tree(acc, width)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        level = to_dev(np.array([len(p) for p in paths], np.int32))
+        rank = to_dev(np.array([p[-1] if p else 0 for p in paths], np.int32))
+        w1, w2 = _heads(shape, 930, len(acc))
+        mw = ghd.MedusaWeights(to_dev(w1), to_dev(w2))
+        gw = ghd.ModelWeights(to_dev(head["embed"]), [gpu_layer_weights(w) for w in layers], to_dev(head["rms_final"]), to_dev(head["lm_head"]))
+        gkv = [ghd.KvLayer(to_dev(k), to_dev(v), ghd.KV_LEN_DEVICE) for k, v in fresh()]
+        ctx = ghd.ghd_create(gpu_cfg(shape, Lmax, width))        # bound to `stream`
+        first_tokens = to_dev(np.array([g[0]] + [0] * (width - 1), np.int32))
+        tok_d = first_tokens.clone()
+        amax = torch.empty(width, dtype=torch.int32, device="cuda")
+        logits_d = torch.empty((width, shape.vocab), dtype=torch.float32, device="cuda")
+        results = torch.zeros((steps, 2 + 2 * ghd.GHD_MAX_NODES), dtype=torch.int32, device="cuda")
+        tree = ghd.Tree(ctx)
+
+        def one_step(s):
+            ghd.ghd_tree_build(ctx, parent, ghd.KV_LEN_DEVICE, tree=tree)
+            ghd.ghd_verify_step(ctx, gw, gkv, tree, tok_d, logits=logits_d, argmax=amax)
+            ghd.ghd_accept(ctx, tree, tok_d, amax, out=results[s])
+            ghd.ghd_kv_commit(ctx, gkv, ghd.KV_LEN_DEVICE, results[s])
+            cand = ghd.ghd_medusa_draft(ctx, mw, results[s], topk)
+            ghd.ghd_tree_fill_tokens(ctx, cand, results[s], level, rank, tokens=tok_d)
+
+        ghd.ghd_kv_len_set(ctx, L0)
+        one_step(0)                                             # warm-up outside the capture (one-time set-up calls)
+        first = logits_d[0].clone()
+        ghd.ghd_sync_status(ctx)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for s in range(steps):
+                one_step(s)
+        for rep in range(2):                                    # the same graph, started twice from the same state
+            ghd.ghd_kv_len_set(ctx, L0)
+            tok_d.copy_(first_tokens)
+            graph.replay()
+            L_end = ghd.ghd_kv_len_get(ctx)
+            ghd.ghd_sync_status(ctx)
+            out = []
+            for r in results.cpu().numpy():
+                out += [int(t) for t in r[258:259 + int(r[0])]]
+            assert steps <= len(out) <= most and L_end == L0 + len(out)
+            assert out == g[1:len(out) + 1]
+    err = np.abs(first.cpu().numpy().astype(np.float64) - first_logits).max()
+    assert err <= tol_for(shape.dtype) * np.abs(first_logits).max()
+    assert min(gaps) > 8.0 * err, "seed gives a near-tie; pick another"
