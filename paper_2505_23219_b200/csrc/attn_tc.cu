@@ -40,6 +40,7 @@ constexpr int QM = 128;        // query rows per CTA (MMA M)
 constexpr int BN = 64;         // keys per unit (MMA N of S, MMA K of PV)
 constexpr int KV_STAGES = 4;
 constexpr int THREADS = 224;
+constexpr int THREADS_DUO = 352;   // two more softmax warpgroups' worth of threads: see k_attn_tc, DUO
 constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 
 struct AttnParams {
@@ -63,11 +64,11 @@ struct AttnSmem {
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
     int abort_flag;
-    float xmax[2][QM];            // row-pair mode: the two threads of a row exchange their partial maxima
-    float xl[QM];                 // ... and, at the end, their partial sums
+    float xmax[2][2 * QM];        // two threads per row: they exchange their partial maxima
+    float xl[2 * QM];             // ... and, at the end, their partial sums
 };
 
-__device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+template <int THREADS_IN> __device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, %0;" ::"n"(THREADS_IN) : "memory"); }
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -79,8 +80,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // query), so S, P and PV come out duplicated and two threads share a row: thread r takes the
 // first 32 keys of a unit and the first half of d_head, thread r + 64 the rest.  This halves the
 // per-unit softmax time, which is what bounds the kernel at small trees.
-template <int DH, bool PAIR>
-__global__ void __launch_bounds__(THREADS, 1)
+// DUO: more than 64 query rows, so nothing can be duplicated; instead a second group of four softmax warps
+// (warps 7..10) shares the tensor-memory lanes of the first (a warp may touch lanes 32 (w mod 4) ..): again two
+// threads per row, the first group's thread taking the first 32 keys of a unit and the first half of d_head.
+template <int DH, bool PAIR, bool DUO = false>
+__global__ void __launch_bounds__(DUO ? THREADS_DUO : THREADS, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
     constexpr int SLABS = DH / 64;                       // 64-wide (128-byte) column slabs of a d_head row
@@ -115,15 +119,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         for (int s = 0; s < KV_STAGES; ++s) { mbar_init(smem_u32(&sm->kv_full[s]), 1); mbar_init(smem_u32(&sm->kv_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sm->s_full[b]), 1);
-            mbar_init(smem_u32(&sm->s_empty[b]), 128);
-            mbar_init(smem_u32(&sm->p_full[b]), 128);
+            mbar_init(smem_u32(&sm->s_empty[b]), DUO ? 256 : 128);
+            mbar_init(smem_u32(&sm->p_full[b]), DUO ? 256 : 128);
             mbar_init(smem_u32(&sm->p_empty[b]), 1);
             mbar_init(smem_u32(&sm->pv_full[b]), 1);
-            mbar_init(smem_u32(&sm->pv_empty[b]), 128);
+            mbar_init(smem_u32(&sm->pv_empty[b]), DUO ? 256 : 128);
         }
         mbar_init(smem_u32(&sm->drain), 1);
         mbar_init(smem_u32(&sm->drain_pv), 1);
-        mbar_init(smem_u32(&sm->mask_ready), 128);
+        mbar_init(smem_u32(&sm->mask_ready), DUO ? 256 : 128);
         for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -293,15 +297,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain_pv), 0); ++spin) __nanosleep(64);
             }
         }
-    } else if constexpr (PAIR) {
+    } else if constexpr (PAIR || DUO) {
         // ------------------------------------------------ softmax warps, two threads per query row
         constexpr int HC = BN / 2;                             // keys of a unit per thread
         constexpr int HD = DH / 2;                             // d_head columns per thread
+        constexpr int NT = DUO ? 256 : 128;                    // softmax threads
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                        // tensor-memory lane
-        const int half = r >> 6, row = r & 63;                 // which half of the row's work, query row
+        // which half of the row's work; the row of the P tile this thread writes; its query row; its exchange slots
+        const int half = DUO ? (warp >= 7 ? 1 : 0) : r >> 6;
+        const int prow_i = DUO ? r : r & 63;
+        const int row = DUO ? row0 + r : r & 63;
+        const int xi = DUO ? half * QM + r : r, xpartner = DUO ? (half ^ 1) * QM + r : r ^ 64;
         const bool live = row < p.n;
-        const bool warp_live = (quad & 1) * 32 < p.n;          // warps whose 32 rows are all padding skip the math
+        const bool warp_live = DUO ? row0 + quad * 32 < p.n : (quad & 1) * 32 < p.n;   // warps whose 32 rows are all padding skip the math
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
         const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain
         pdl_wait();                                            // the mask comes from an earlier kernel
@@ -363,7 +372,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
             if (!warp_live) {
                 mbar_arrive(smem_u32(&sm->s_empty[b]));
-                pair_bar();                                    // every softmax thread takes part in the exchange barrier
+                pair_bar<NT>();                                // every softmax thread takes part in the exchange barrier
                 if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 mbar_arrive(smem_u32(&sm->p_full[b]));
                 if (i >= 1) fold_pv(i - 1, 1.f);
@@ -385,15 +394,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
             }
             const float mine = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            sm->xmax[b][r] = mine;                             // the partner thread (lane r ^ 64) holds the other 32 keys
-            pair_bar();
-            const float tmax = fmaxf(mine, sm->xmax[b][r ^ 64]) * sl2;
+            sm->xmax[b][xi] = mine;                            // the partner thread holds the other 32 keys
+            pair_bar<NT>();
+            const float tmax = fmaxf(mine, sm->xmax[b][xpartner]) * sl2;
             const float m_new = fmaxf(m, tmax);
             const float neg = (m_new == -INFINITY) ? 0.f : -m_new;
             const float corr = (m_new == -INFINITY) ? 1.f : ex2_approx(m + neg);
             if (i >= 2) mbar_wait(smem_u32(&sm->p_empty[b]), ((i >> 1) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
-            // this thread's 32 probabilities go into both copies of the row (tile rows row and row + 64)
-            uint8_t* prow = p_ptr + b * P_BYTES + row * 128;
+            // this thread's 32 probabilities go into the row (PAIR: into both copies, tile rows row and row + 64)
+            uint8_t* prow = p_ptr + b * P_BYTES + prow_i * 128;
             float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -407,10 +416,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     const __half2 hh = __floats2half2_rn(p0, p1);
                     packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
                 }
-                const uint32_t off = (uint32_t)(((half * 4 + q) ^ (row & 7)) << 4);
+                const uint32_t off = (uint32_t)(((half * 4 + q) ^ (prow_i & 7)) << 4);
                 const uint4 val = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                 *reinterpret_cast<uint4*>(prow + off) = val;
-                *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
+                if constexpr (!DUO) *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(smem_u32(&sm->p_full[b]));
@@ -421,8 +430,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             return true;
         });
         if (cnt > 0) fold_pv(cnt - 1, corr_prev);
-        sm->xl[r] = l;
-        pair_bar();
+        sm->xl[xi] = l;
+        pair_bar<NT>();
         if (live) {
             float* po = p.part_o + ((size_t)split * p.max_nodes + row) * (size_t)(p.heads * DH) + h * DH + half * HD;
 #pragma unroll
@@ -430,7 +439,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             if (half == 0) {
                 float* pm = p.part_ml + (((size_t)split * p.max_nodes + row) * p.heads + h) * 2;
                 pm[0] = m * 0.6931471805599453f;               // back to the natural-log domain the merge kernel uses
-                pm[1] = l + sm->xl[r ^ 64];
+                pm[1] = l + sm->xl[xpartner];
             }
         }
     } else {
@@ -616,18 +625,23 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         if (cudaFuncSetAttribute(k_attn_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess ||
-            cudaFuncSetAttribute(k_attn_tc<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess) {
+            cudaFuncSetAttribute(k_attn_tc<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b64) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b128) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 attention: cannot raise dynamic shared memory");
             cudaGetLastError();
             return GHD_ECUDA;
         }
         c->attr_attn = true;
     }
+    const bool duo = !pair && c->opt_attn_rows != 1;     // more than 64 rows: two softmax warpgroups share the rows
     if (dh == 64) {
         if (pair) launch_k(c, true, k_attn_tc<64, true>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
+        else if (duo) launch_k(c, true, k_attn_tc<64, false, true>, grid, THREADS_DUO, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
         else launch_k(c, true, k_attn_tc<64, false>, grid, THREADS, attn_smem_bytes<64>(), tm_q, tm_k, tm_v, p);
     } else {
         if (pair) launch_k(c, true, k_attn_tc<128, true>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
+        else if (duo) launch_k(c, true, k_attn_tc<128, false, true>, grid, THREADS_DUO, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
         else launch_k(c, true, k_attn_tc<128, false>, grid, THREADS, attn_smem_bytes<128>(), tm_q, tm_k, tm_v, p);
     }
     if (coo) launch_attn_coo(c, q, kv, t, splits);       // the sparse part as one more partial, slot `splits`
