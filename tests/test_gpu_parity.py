@@ -564,6 +564,39 @@ def test_small_step_logits_argmax_accept(ghd, shape, graph):
     assert np.array_equal(res[2:3 + m], nodes) and np.array_equal(res[258:259 + m], toks)
 
 
+@pytest.mark.parametrize("n", [24, 64, 130, 200])
+def test_step_is_bit_reproducible_across_reruns_and_launch_modes(ghd, n):
+    """Fixed reduction orders everywhere (split tiles in worker order, KV splits in split order): the same step gives
+    the same bits when it is run again, replayed from the library's graph, or run with the norms in the epilogues twice."""
+    shape, L = SMALL16_DH128, 90
+    Lmax = L + n
+    parent = wl.random_tree(n, 6, 811 + n, max_children=4)
+    tokens = wl.draft_tokens(parent, shape.vocab, 812 + n)
+    head, layers, caches, gw, _ = _model(ghd, shape, 13, L, Lmax)
+    tok_d = to_dev(tokens)
+
+    def run(opts, graph, reps):
+        ctx = make_ctx(ghd, shape, Lmax, n)
+        for o, v in opts:
+            ghd.ghd_set_option(ctx, o, v)
+        ghd.ghd_set_option(ctx, ghd.OPT_GRAPH, graph)
+        tree = ghd.ghd_tree_build(ctx, parent, L)
+        outs = []
+        for _ in range(reps):
+            gkv = [ghd.KvLayer(to_dev(k), to_dev(v), L) for k, v in caches]
+            logits, amax = ghd.ghd_verify_step(ctx, gw, gkv, tree, tok_d)
+            ghd.ghd_sync_status(ctx)
+            outs.append((logits.cpu().numpy().copy(), gkv[-1].k.cpu().numpy().copy()))
+        return outs
+
+    direct = run([], 0, 2)
+    replay = run([], 2, 2)
+    for lg, kc in direct[1:] + replay:
+        assert np.array_equal(lg, direct[0][0]) and np.array_equal(kc, direct[0][1])
+    fused = run([(ghd.OPT_FUSED_NORM, 1)], 0, 2)
+    assert np.array_equal(fused[0][0], fused[1][0]) and np.array_equal(fused[0][1], fused[1][1])
+
+
 def test_width1_chain_reproduces_sequential_greedy_steps_on_gpu(ghd):
     shape, k, L = SMALL32, 5, 30
     Lmax = L + k + 1
