@@ -73,6 +73,8 @@ typedef enum ghd_option {
                                  than 128 nodes, 1 = never, 2 = whenever the shape allows (even tile count)          */
     GHD_OPT_ATTN_ROWS = 13,   /* tcgen05 attention, trees of more than 64 nodes: 0 = two softmax threads per query row
                                  (two groups of four warps on the same tensor-memory lanes), 1 = one thread per row     */
+    GHD_OPT_GEMM_SKEW = 14,   /* tcgen05 GEMM with three CTAs per two tiles: k-chunks taken from the middle CTA of every
+                                 group (0 = automatic, 1 = none, s + 1 = s chunks), so that it is done before its neighbours */
     GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
                                  Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
                                  nobody sees them (default); 1 = per-query list of visible nodes (the

@@ -12,10 +12,11 @@
 // and cut into equal contiguous ranges, one per CTA (one CTA per SM), so every SM
 // streams the same number of weight bytes whatever the tile count.  A CTA whose
 // range covers only part of a tile's k-steps writes its float partial tile to the
-// workspace and bumps the tile's arrival counter; the tile's first contributor (for
-// which the tile comes last) keeps its share in tensor memory, waits - bounded - for
-// that counter, sums the partials in CTA order (fixed order -> bit-reproducible) and
-// runs the epilogue.  Contributors that store never wait.
+// workspace and bumps the tile's arrival counter; the contributor that completes its
+// share of the tile last (chosen on the host from the ranges) keeps that share in
+// tensor memory, waits - bounded - for the counter, adds the others' partials in CTA
+// order (fixed order -> bit-reproducible) and runs the epilogue.  Contributors that
+// store never wait.
 //
 // Per CTA: warp 0 = TMA producer (weights and activations into a ring of
 // 128B-swizzled shared-memory stages), warp 1 = MMA issuer (tcgen05.mma, one
@@ -63,9 +64,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
     const int rank = PAIR ? (int)cluster_ctarank() : 0;      // 0: the CTA that issues the pair's MMAs
-    const int G = PAIR ? gridDim.x / 2 : gridDim.x, wk = PAIR ? cta >> 1 : cta;     // workers and this CTA's worker
-    const long long total = (long long)p.n_work * p.kiters;
-    const long long it_beg = total * wk / G, it_end = total * (wk + 1) / G;
+    const int wk = PAIR ? cta >> 1 : cta;                   // this CTA's worker: a CTA, or a pair of CTAs
+    const long long it_beg = p.range_beg[wk], it_end = p.range_beg[wk + 1];
     const int my_iters = (int)(it_end - it_beg);
     const int prefill = my_iters < p.stages ? my_iters : p.stages;    // weight stages requested during set-up
     // work unit -> this CTA's 128-row tile, and the row coordinate of that tile in the weight map
@@ -254,13 +254,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         // Epilogue of a complete tile.  split = false: the accumulator holds the whole sum.  split = true: this CTA
         // (the tile's first contributor) has its share in tensor memory and adds the other contributors' partial
         // tiles from the workspace in worker order (fixed order -> reproducible); each one's 32 loads go out together.
-        auto finish_tile = [&](int tile_, uint32_t t_addr_, bool split, int c_first_, int c_last_) {
+        auto finish_tile = [&](int wt_, int tile_, uint32_t t_addr_, bool split, int c_first_, int c_last_) {
             for (int c0 = grp * EPI_CHUNK; c0 < p.nb && c0 < p.n; c0 += GROUPS * EPI_CHUNK) {
                 float v[32];
                 tc_ld32(t_addr_ + c0, v);                  // may run past nb, never past the buffer
                 if (split) {
-                    for (int c = c_first_ + 1; c <= c_last_; ++c) {      // later contributors always use their slot 0
-                        const float* src = part_of(c) + (size_t)c0 * TILE_M + row;
+                    for (int c = c_first_; c <= c_last_; ++c) {          // the first contributor's slot varies, later ones use slot 0
+                        if (c == wk) continue;                             // this CTA's own share came from tensor memory
+                        const float* src = part_of(c) + (size_t)(c == c_first_ ? p.tile_slot[wt_] * slot_elems : 0) + (size_t)c0 * TILE_M + row;
                         float t[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) t[j] = __ldcg(src + (size_t)j * TILE_M);
@@ -311,19 +312,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + buf * buf_cols + ((uint32_t)(quad * 32) << 16);
-            // A tile some workers share is finished by its FIRST contributor: for that CTA the tile is the last unit of
-            // its range, so it gets here last in time, while every other contributor handles its share as the first
-            // unit of its range (or as its only one), stores it and counts itself in without ever waiting.  The
-            // finisher keeps its own share in tensor memory and waits (bounded) for the others; they run at the same
-            // time on other SMs and depend on nobody, so the wait is short: the store and count of a contributor
-            // that ended together with the finisher.
+            // A tile some workers share is finished by the contributor that completes its share of it LAST (the host
+            // knows from the ranges: usually the first contributor, for which the tile is the last unit of its range,
+            // while every other contributor handles its share as the first unit of its range, stores it and counts
+            // itself in without ever waiting).  The finisher keeps its own share in tensor memory and waits (bounded)
+            // for the others; they run at the same time on other SMs and depend on nobody, so the wait is short.
             const int c_first = p.tile_first[wt], c_last = c_first + p.tile_count[wt] - 1;
             bool finish = whole;
             if (!whole && sliced) pend_wt[n_pend++] = wt;
             if (!whole && p.epi.mode != EPI_DEFER && !sliced) {
                 if (et == 0) {
                     int fl = 0;
-                    if (wk == c_first) {
+                    if (wk == c_first + p.tile_fin[wt]) {
                         fl = 1;
                         uint32_t spin = 0;
                         while (ld_acquire_gpu(p.counters + tile) != c_last - c_first) {
@@ -338,7 +338,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 epi_all();
             }
             if (finish) {
-                finish_tile(tile, t_addr, !whole, c_first, c_last);
+                finish_tile(wt, tile, t_addr, !whole, c_first, c_last);
                 if (!whole && et == 0) p.counters[tile] = 0;   // ready for the next launch
             } else {
                 // partial tile: slot 0 when this is the CTA's first unit (it starts mid-tile or is
@@ -556,13 +556,40 @@ ghd_status plan_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, 
     const int ctas = workers * per;
     p.ctas = ctas;
     plan->smem = smem_bytes_for(nb_cta, p.ks, p.stages);
+    if (workers > MAX_WORKERS) {
+        snprintf(c->err, sizeof(c->err), "tcgen05 GEMM: more than %d workers", MAX_WORKERS);
+        return GHD_EUNSUPPORTED;
+    }
+    for (int w2 = 0; w2 <= workers; ++w2) p.range_beg[w2] = (int)(total * w2 / workers);
+    // Three workers per two work units (every range 2/3 of a unit): the middle worker of a group holds the tail of one
+    // unit and the head of the next and would end together with the worker that finishes the second unit, which would
+    // then wait for its store.  A few k-chunks less for the middle worker and it is done early; the outer two grow a
+    // little and each finishes its own unit without waiting.
+    int skew = c->opt_gemm_skew > 0 ? c->opt_gemm_skew - 1 : 1;       // automatic: one k-chunk, as measured
+    if (epi.mode != EPI_DEFER && workers % 3 == 0 && (long long)workers * 2 == (long long)p.n_work * 3 && skew > 0 && 3 * skew < p.kiters)
+        for (int g = 0; g < workers / 3; ++g) {
+            p.range_beg[3 * g + 1] += skew;          // the first worker of the group takes `skew` more
+            p.range_beg[3 * g + 2] -= skew;          // so does the third
+        }
     for (int t = 0; t < p.n_work; ++t) {
-        const long long t_first = (long long)t * p.kiters;
-        const int c_first = (int)(((t_first + 1) * workers + total - 1) / total) - 1;
-        const int c_last = (int)(((t_first + p.kiters) * workers + total - 1) / total) - 1;
+        const long long t_first = (long long)t * p.kiters, t_end = t_first + p.kiters;
+        int c_first = 0;
+        while (p.range_beg[c_first + 1] <= t_first) ++c_first;
+        int c_last = c_first;
+        while (c_last + 1 < workers && p.range_beg[c_last + 1] < t_end) ++c_last;
         p.tile_first[t] = (unsigned short)c_first;
         p.tile_count[t] = (unsigned char)(c_last - c_first + 1);
-        p.tile_slot[t] = (total * c_first / workers >= t_first) ? 0 : 1;
+        p.tile_slot[t] = (p.range_beg[c_first] >= t_first) ? 0 : 1;
+        // the finisher: the contributor that completes its share of this tile last, counted in k-chunks from the start
+        // of its own range (all workers start together); the first contributor on a tie: for it the tile comes last
+        auto share_done = [&](int cc) {
+            const long long e = p.range_beg[cc + 1] < t_end ? p.range_beg[cc + 1] : t_end;
+            return e - p.range_beg[cc];
+        };
+        int fin = c_first;
+        for (int cc = c_first + 1; cc <= c_last; ++cc)
+            if (share_done(cc) > share_done(fin)) fin = cc;
+        p.tile_fin[t] = (unsigned char)(fin - c_first);
     }
     plan->pending.active = 0;
     if (epi.mode == EPI_DEFER) {

@@ -16,6 +16,7 @@ constexpr int EPI_CHUNK = 32;        // accumulator columns per tcgen05.ld
 constexpr int THREADS = 192;
 constexpr int THREADS_TC = 320;      // k_gemm_tc: producer warp, MMA warp, two groups of four epilogue warps
 constexpr int MAX_TILES = 256;
+constexpr int MAX_WORKERS = 256;    // CTAs (or CTA pairs) of one launch
 constexpr int DONE_OFF = 2048;       // counters[DONE_OFF + tile]: contributors that have finished their slice of a split tile
 
 struct GemmParams {
@@ -33,6 +34,10 @@ struct GemmParams {
     // worker, number of contributors, slot of the first contributor (the others use slot 0)
     unsigned short tile_first[MAX_TILES];
     unsigned char tile_count[MAX_TILES], tile_slot[MAX_TILES];
+    unsigned char tile_fin[MAX_TILES];   // which contributor (offset from the first) finishes a split tile: the one that ends last
+    // first (work unit, k-chunk) iteration of every worker, and the end of the last: equal shares, except where the
+    // host skews them so that the contributors of a tile do not all end together
+    int range_beg[MAX_WORKERS + 1];
 };
 
 using namespace tc;

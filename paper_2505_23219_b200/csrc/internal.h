@@ -83,7 +83,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm, opt_gemm_pair, opt_attn_rows;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm, opt_gemm_pair, opt_attn_rows, opt_gemm_skew;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
