@@ -19,7 +19,7 @@ __all__ = [
     "ghd_verify_step", "ghd_accept", "ghd_linear", "ghd_rmsnorm", "ghd_tree_attention", "ghd_argmax",
     "ghd_sync_status", "ghd_launch_count", "pack_mask", "ghd_copy_hidden", "ghd_gate_up", "ghd_tree_attention_static", "ghd_path_count", "ghd_kv_commit", "ghd_medusa_draft", "ghd_tree_fill_tokens",
     "ghd_kv_len_set", "ghd_kv_len_get", "KV_LEN_DEVICE", "MedusaWeights", "GHD_MAX_TOPK",
-    "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_ATTN_COO", "PATH_GEMM_PAIR", "OPT_GEMM_PAIR", "OPT_ATTN_ROWS", "OPT_GEMM_SKEW",
+    "PATH_GEMM_TILE", "PATH_GEMM_SIMT", "PATH_ATTN_TC", "PATH_ATTN_SIMT", "PATH_ATTN_COO", "PATH_GEMM_PAIR", "OPT_GEMM_PAIR", "OPT_ATTN_ROWS", "OPT_GEMM_SKEW", "OPT_ATTN_SMALL",
     "GHD_F32", "GHD_F16", "GHD_MAX_NODES", "OPT_GEMM_PATH", "OPT_ATTN_SPLITS", "OPT_ATTN_PATH", "OPT_GRAPH",
     "OPT_GEMM_CTAS", "OPT_GEMM_BURST", "OPT_NO_PDL", "OPT_GEMM_STAGES", "OPT_GEMM_EPI", "OPT_ATTN_SPARSE", "OPT_CHAIN_CALLS", "OPT_FUSED_NORM", "EXPORTS",
 ]
@@ -31,7 +31,7 @@ KV_LEN_DEVICE = -1      # "take the cache length from the context's device word"
 OPT_GEMM_PATH, OPT_ATTN_SPLITS, OPT_ATTN_PATH, OPT_GRAPH, OPT_GEMM_CTAS, OPT_GEMM_BURST, OPT_NO_PDL = 0, 1, 2, 3, 4, 5, 6
 OPT_GEMM_STAGES, OPT_GEMM_EPI, OPT_ATTN_SPARSE, OPT_CHAIN_CALLS, OPT_FUSED_NORM = 7, 8, 9, 10, 11
 PATH_GEMM_TILE, PATH_GEMM_SIMT, PATH_ATTN_TC, PATH_ATTN_SIMT, PATH_ATTN_COO, PATH_GEMM_PAIR = 0, 1, 2, 3, 4, 5
-OPT_GEMM_PAIR, OPT_ATTN_ROWS, OPT_GEMM_SKEW = 12, 13, 14
+OPT_GEMM_PAIR, OPT_ATTN_ROWS, OPT_GEMM_SKEW, OPT_ATTN_SMALL = 12, 13, 14, 15
 _STATUS = ["GHD_OK", "GHD_EINVAL", "GHD_ESHAPE", "GHD_ETREE", "GHD_ENOSPACE", "GHD_ECUDA", "GHD_ETIMEOUT",
            "GHD_EUNSUPPORTED"]
 

@@ -596,6 +596,17 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: operands must be 16-byte aligned");
         return GHD_EINVAL;
     }
+    // The small-tree kernel with 128-key units: as measured it wins on mid-sized trees over a long cache (64 nodes:
+    // -1.3 us at KV 2048, -1.9 us at KV 4096) and loses on short caches or tiny trees (+1 us at KV 512).
+    const bool small = c->opt_attn_small == 1 || (c->opt_attn_small == 0 && n > 32 && kv_len_host_of(c, t) >= 1024);
+    if (n <= 64 && small) {
+        ghd_status st;
+        const int s = launch_attn_tc_small(c, q, kv, t, coo, &st);
+        if (s <= 0) return st;
+        if (coo) launch_attn_coo(c, q, kv, t, s);
+        launch_attn_combine(c, out, s + (coo ? 1 : 0), n);
+        return GHD_OK;
+    }
     CUtensorMap tm_q, tm_k, tm_v;
     const bool pair = n <= 64;                           // two threads per query row (queries loaded twice)
     if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, pair ? 64 : QM, &tm_q) ||

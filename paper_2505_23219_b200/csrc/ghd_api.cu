@@ -245,7 +245,7 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->cap_stream = nullptr;
     c->device = dev;
     c->sm_count = sms;
-    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = c->opt_chain_calls = c->opt_fused_norm = c->opt_gemm_pair = c->opt_attn_rows = c->opt_gemm_skew = 0;
+    c->opt_gemm_path = c->opt_attn_splits = c->opt_attn_path = c->opt_graph = c->opt_gemm_ctas = c->opt_gemm_burst = c->opt_no_pdl = c->opt_gemm_stages = c->opt_gemm_epi = c->opt_attn_sparse = c->opt_chain_calls = c->opt_fused_norm = c->opt_gemm_pair = c->opt_attn_rows = c->opt_gemm_skew = c->opt_attn_small = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->max_splits = 16;
@@ -253,7 +253,7 @@ ghd_status ghd_create(const ghd_model_cfg* cfg, void* cuda_stream, ghd_ctx** out
     c->h_ssq = -1;
     c->kv_len_hint = 0;
     c->entry_fresh = c->opt_chain_calls ? 0 : 1;
-    c->attr_gemm = c->attr_attn = false;
+    c->attr_gemm = c->attr_attn = c->attr_attn_small = false;
     c->launches = 0;
     memset(c->path_count, 0, sizeof(c->path_count));
     c->tmaps = new std::map<TmapKey, std::vector<uint64_t>>();
@@ -305,6 +305,7 @@ ghd_status ghd_set_option(ghd_ctx* c, int32_t option, int32_t value) {
         case GHD_OPT_GEMM_PAIR: if (value > 2) return GHD_EINVAL; c->opt_gemm_pair = value; break;
         case GHD_OPT_ATTN_ROWS: if (value > 1) return GHD_EINVAL; c->opt_attn_rows = value; break;
         case GHD_OPT_GEMM_SKEW: if (value > 64) return GHD_EINVAL; c->opt_gemm_skew = value; break;
+        case GHD_OPT_ATTN_SMALL: if (value > 2) return GHD_EINVAL; c->opt_attn_small = value; break;
         case GHD_OPT_ATTN_SPARSE: if (value > 1) return GHD_EINVAL; c->opt_attn_sparse = value; break;
         case GHD_OPT_GEMM_EPI: if (value > 2) return GHD_EINVAL; c->opt_gemm_epi = value; break;
         case GHD_OPT_GEMM_BURST: if (value > 8) return GHD_EINVAL; c->opt_gemm_burst = value; break;
@@ -417,7 +418,7 @@ ghd_status ghd_verify_step(ghd_ctx* c, const ghd_model_weights* w, ghd_kv_layer*
     push(w->embed); push(w->rms_final); push(w->lm_head); push(tokens_dev); push(logits); push(argmax_dev);
     push(tree->mask); push(tree->depth); push(tree->pos); push(tree->rope); push(tree->coo_ptr); push(tree->coo_col);
     key.push_back(((uint64_t)(uint32_t)tree->n << 32) | (uint32_t)tree->kv_len);
-    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse, c->opt_chain_calls, c->opt_fused_norm, c->opt_gemm_pair, c->opt_attn_rows, c->opt_gemm_skew})
+    for (int o : {c->opt_gemm_path, c->opt_attn_splits, c->opt_attn_path, c->opt_gemm_ctas, c->opt_gemm_burst, c->opt_no_pdl, c->opt_gemm_stages, c->opt_gemm_epi, c->opt_attn_sparse, c->opt_chain_calls, c->opt_fused_norm, c->opt_gemm_pair, c->opt_attn_rows, c->opt_gemm_skew, c->opt_attn_small})
         key.push_back((uint64_t)(uint32_t)o);       // every option that changes what is enqueued
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const ghd_layer_weights& lw = w->layers[l];

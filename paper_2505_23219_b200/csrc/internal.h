@@ -83,7 +83,7 @@ struct ghd_ctx {
     cudaStream_t cap_stream;  // library-owned stream used only for graph capture (nothing ever runs on it)
     int device, sm_count;
     // options
-    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm, opt_gemm_pair, opt_attn_rows, opt_gemm_skew;
+    int opt_gemm_path, opt_attn_splits, opt_attn_path, opt_graph, opt_gemm_ctas, opt_gemm_burst, opt_no_pdl, opt_gemm_stages, opt_gemm_epi, opt_attn_sparse, opt_chain_calls, opt_fused_norm, opt_gemm_pair, opt_attn_rows, opt_gemm_skew, opt_attn_small;
     // workspace carve (all device pointers into the caller's buffer)
     char* ws;
     size_t ws_bytes;
@@ -109,7 +109,7 @@ struct ghd_ctx {
     ghd::PendingPartials pending;   // projection output not yet folded into xres
     // bookkeeping
     int entry_fresh;          // 1 until the first launch of a public call: that launch is fully serialised (see launch_k)
-    bool attr_gemm, attr_attn;  // dynamic shared memory limits raised on this context's device
+    bool attr_gemm, attr_attn, attr_attn_small;  // dynamic shared memory limits raised on this context's device
     int64_t launches;
     int64_t path_count[8];   // launches per kernel family (ghd_path)
     char err[256];
@@ -222,6 +222,9 @@ bool attn_tc_supported(const ghd_ctx* c, const ghd_tree* t);
 // the split partials go to att_o / att_ml and a second kernel merges them into `out`
 // coo: the new rows are handled by launch_attn_coo (one more partial), this kernel takes the cache only
 ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, void* out, bool coo);
+// attn_tc_small.cu : the split kernel for trees of up to 64 nodes (128-key units, accumulator resident in tensor
+// memory); leaves the partials in att_o / att_ml and returns the number of splits (0 and *st after an error)
+int launch_attn_tc_small(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, const ghd_tree* t, bool coo, ghd_status* st);
 
 // gemm_tc.cu : tcgen05 / TMA path (GHD_F16 only)
 ghd_status launch_gemm_tc(ghd_ctx* c, const void* x, const void* w, int n, int k, int m, const EpiArgs& epi);

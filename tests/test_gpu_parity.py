@@ -211,12 +211,14 @@ def test_small_layers_with_projections_on_cta_pairs(ghd, n, L):
     assert ghd.ghd_path_count(ctx, ghd.PATH_GEMM_PAIR) >= (3 if n > 16 else 0)     # QKV, O, down (gate/up has 11 tiles)
 
 
-def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0, on_device=False):
+def _attention_case(ghd, shape, n, L, parent, splits, seed=400, path=0, sparse=0, on_device=False, opts=()):
     Lmax = L + n + (150 if on_device else 3)               # on_device: the kernels see cache rows far past kv_len + n
     ctx = make_ctx(ghd, shape, Lmax, max(n, 8))
     if path:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_PATH, path)
     ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPARSE, sparse)
+    for o, v in opts:
+        ghd.ghd_set_option(ctx, o, v)
     if splits:
         ghd.ghd_set_option(ctx, ghd.OPT_ATTN_SPLITS, splits)
     H, dh, dt = shape.n_heads, shape.d_head, shape.dtype
@@ -274,10 +276,31 @@ def test_tree_attention_with_the_cache_length_on_the_device(ghd, shape, n, L, sp
         assert _attention_case(ghd, shape, n, L, parent, splits, path=1, on_device=True) <= tol
 
 
+@pytest.mark.parametrize("shape", [SMALL16, SMALL16_DH128], ids=["f16", "f16dh128"])
+@pytest.mark.parametrize("n,L,splits", [(1, 0, 0), (1, 1, 1), (8, 256, 0), (9, 63, 1), (33, 65, 3), (64, 300, 0), (64, 300, 16), (64, 2048, 0),
+                                        (49, 640, 5), (17, 129, 2), (64, 127, 0), (40, 4096, 0)])
+def test_tree_attention_small_tree_kernel_with_128_key_units(ghd, shape, n, L, splits):
+    """GHD_OPT_ATTN_SMALL: 128-key units, output accumulator resident in tensor memory (rescaled in place when the
+    reference maximum rises); plain, with the coordinate index for the new rows, and with the cache length on the device."""
+    parent = wl.random_tree(n, 8, 1000 + n, max_children=6)
+    small = [(ghd.OPT_ATTN_SMALL, 1)]
+    assert _attention_case(ghd, shape, n, L, parent, splits, opts=small) <= 2e-3
+    assert _attention_case(ghd, shape, n, L, parent, splits, sparse=1, opts=small) <= 2e-3
+    assert _attention_case(ghd, shape, n, L, parent, splits, on_device=True, opts=small) <= 2e-3
+    assert _attention_case(ghd, wl.scaled(shape, name="chain"), n, L, wl.chain_tree(n), splits, opts=small) <= 2e-3
+
+
+@pytest.mark.parametrize("n,L", [(1, 40), (13, 100), (64, 77)])
+def test_small_layers_with_the_small_tree_attention_kernel(ghd, n, L):
+    import paper_2505_23219_b200 as g
+    _layer_case(ghd, SMALL16_DH128, 11, n, L, wl.random_tree(n, 8, 40 + n, max_children=6), opts=[(g.OPT_ATTN_SMALL, 1)])
+
+
 @pytest.mark.parametrize("n,L,splits", [(64, 2048, 0), (64, 2048, 5), (200, 1000, 0), (256, 4096, 0), (49, 640, 3)])
 def test_tree_attention_long_cache_both_paths(ghd, n, L, splits):
     parent = wl.random_tree(n, 8, 2000 + n, max_children=6)
-    assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits) <= 2e-3               # tcgen05 kernel
+    assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits) <= 2e-3               # tcgen05 kernel (automatic choice)
+    assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits, opts=[(ghd.OPT_ATTN_SMALL, 2)]) <= 2e-3   # 64-key units
     assert _attention_case(ghd, SMALL16_DH128, n, L, parent, splits, path=1) <= 2e-3       # CUDA-core kernel
 
 
