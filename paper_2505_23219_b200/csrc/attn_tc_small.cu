@@ -1,8 +1,11 @@
 // Tree attention for trees of up to 64 nodes on the tensor cores (sm_100a, half in, float softmax/accumulate):
 // the small-tree shape of k_attn_tc with 128-key units and the output accumulator kept in tensor memory.
 //
-// One CTA = one head x one KV split.  The queries (at most 64 rows) are loaded twice, so that two threads share
-// a query row: thread r takes the first 64 keys of a unit and the first half of d_head, thread r + 64 the rest.
+// One CTA = one head x one KV split.  FOUR threads share a query row: the queries (at most 64 rows) are loaded
+// twice (tile rows r and r + 64 hold the same query; the copy picks a 64-key half of a unit and a half of d_head)
+// and two groups of four softmax warps work on the same tensor-memory lanes (the group picks 32 of those 64 keys).
+// The per-unit softmax work of a thread - one 32-column read of S, 32 exponentials, four 16-byte stores of P - is
+// what the unit chain waits for, so spreading it over 256 threads shortens every unit.
 // Keys are walked in 128-key units: the cache rows [0, kv_len) first (the dense part), then the new rows as one
 // group of up to 128 nodes (the sparse part, masked by the packed ancestor bitmask; dropped when no query of the
 // CTA sees any of them).  Every unit costs a fixed chain of hand-overs between the asynchronous units
@@ -13,8 +16,9 @@
 // K and V tiles of a unit travel separately (K is free again after S, V after PV).
 //
 // The un-normalised (o, max, sum) of a split go to the workspace; k_attn_combine_rows merges the splits
-// (paper Sec. III-B-2).  Warp 0 = TMA producer, warp 1 = issuer of the S MMAs + tensor-memory owner, warps 2..5 =
-// softmax (128 threads = 128 tensor-memory lanes), warp 6 = issuer of the PV MMAs.  All waits are bounded.  Cache
+// (paper Sec. III-B-2).  Warp 0 = TMA producer, warp 1 = issuer of the S MMAs + tensor-memory owner, warps 2..5 and
+// 7..10 = softmax (a warp may touch the tensor-memory lanes 32 (w mod 4) ..), warp 6 = issuer of the PV MMAs.  All
+// waits are bounded.  Cache
 // tiles that lie wholly below kv_len cannot be touched by the preceding kernel, so the producer requests the first
 // of them, and asks the L2 for the rest, before it waits for that kernel to finish.
 #include <cstdio>
@@ -29,7 +33,7 @@ namespace {
 using namespace tc;
 
 constexpr int QM = 128;        // query rows per CTA (MMA M)
-constexpr int THREADS = 224;
+constexpr int THREADS = 352;       // producer, S issuer, four softmax warps, PV issuer, four more softmax warps
 constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 constexpr int NODE_WEIGHT = 2;     // cost of a node-group unit in cache-tile units, for the split of a head
 constexpr int CTRL_BYTES = 1536;   // control block behind the tiles
@@ -75,15 +79,15 @@ struct AttnSmem {
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];   // K and V tiles of a unit travel separately: K is free again after S, V after PV
     uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2], pv_full[2], pv_empty[2];
     uint64_t drain, drain_pv;
-    uint64_t mask_ready;          // all 128 row threads have merged their mask words into word_or
+    uint64_t mask_ready;          // all softmax threads have merged their mask words into word_or
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
     int abort_flag;
-    float xch[2][QM];             // row-pair mode: the two threads of a row exchange their partial maxima (slot = unit parity) and, at the end, sums
+    float xch[2][QM];             // the four threads of a row exchange their partial maxima and, at the end, sums: [warp group][lane]
 };
 static_assert(sizeof(AttnSmem) <= CTRL_BYTES, "control block too large");
 
-__device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+__device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, 256;" ::: "memory"); }     // all softmax threads
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -145,15 +149,15 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sm->s_full[b]), 1);
-            mbar_init(smem_u32(&sm->s_empty[b]), 128);
-            mbar_init(smem_u32(&sm->p_full[b]), 128);
+            mbar_init(smem_u32(&sm->s_empty[b]), 256);
+            mbar_init(smem_u32(&sm->p_full[b]), 256);
             mbar_init(smem_u32(&sm->p_empty[b]), 1);
             mbar_init(smem_u32(&sm->pv_full[b]), 1);
-            mbar_init(smem_u32(&sm->pv_empty[b]), 128);
+            mbar_init(smem_u32(&sm->pv_empty[b]), 256);
         }
         mbar_init(smem_u32(&sm->drain), 1);
         mbar_init(smem_u32(&sm->drain_pv), 1);
-        mbar_init(smem_u32(&sm->mask_ready), 128);
+        mbar_init(smem_u32(&sm->mask_ready), 256);
         for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -383,12 +387,17 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 for (uint32_t spin = 0; spin < SPIN_LIMIT && !mbar_try(smem_u32(&sm->drain_pv), 0); ++spin) __nanosleep(64);
             }
         }
-    } else if (warp >= 2 && warp <= 5) {
+    } else if ((warp >= 2 && warp <= 5) || warp >= 7) {
         // ------------------------------------------------ softmax warps
-        // two threads per query row (thread r: keys [0, 64) of a unit and the first half of d_head; thread r + 64: the rest)
-        constexpr int HC = 64;                                 // keys of a unit per thread: half of the unit's 128
-        static_assert(BN / 2 == HC, "a thread takes 64 keys of a unit");
-        constexpr int HD = DH / 2;                             // d_head columns per thread
+        // FOUR threads per query row.  The tile rows r and r + 64 hold the same query (half = r / 64 picks the 64-key
+        // half of a unit and the half of d_head), and two groups of four warps (warps 2..5 and 7..10) work on the same
+        // tensor-memory lanes (grp picks 32 of those 64 keys and, when the accumulator is rescaled, half of its columns).
+        constexpr int HC = 32;                                 // keys of a unit per thread: a quarter of the unit's 128
+        static_assert(BN / 4 == HC, "a thread takes 32 keys of a unit");
+        constexpr int HD = DH / 2;                             // d_head columns per row copy
+        constexpr int OC = HD >= 64 ? HD / 2 : HD;             // output columns a thread carries home at the end
+        const int grp = warp >= 7 ? 1 : 0;
+        const bool carries = HD >= 64 || grp == 0;             // (d_head 64: the first group takes all 32 columns of its half)
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                        // tensor-memory lane
         const int half = r >> 6;
@@ -425,35 +434,30 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
             }
             const int cnt = walk([&](int i, int key0, int g) -> bool {
                 const int b = i & 1, pb = i % P_BUFS;
-                unsigned long long vis = 0ull;                 // visibility of this thread's 64 keys of the unit
+                uint32_t vis = 0u;                             // visibility of this thread's 32 keys of the unit
                 if (g < 0) {
-                    const int valid = kv_len - key0 - half * HC;
-                    if (live) vis = valid >= 64 ? ~0ull : (valid > 0 ? ((1ull << valid) - 1ull) : 0ull);
+                    const int valid = kv_len - key0 - half * 64 - grp * HC;
+                    if (live) vis = valid >= HC ? 0xffffffffu : (valid > 0 ? ((1u << valid) - 1u) : 0u);
                 } else if (g * KSL + half == 0) {
-                    vis = myw[0];                              // up to 64 nodes: only word 0 exists
+                    vis = (uint32_t)(myw[0] >> (grp * HC));    // up to 64 nodes: only word 0 exists
                 }
                 mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 if (!warp_live) {
                     mbar_arrive(smem_u32(&sm->s_empty[b]));
-                    pair_bar();                                // every softmax thread takes part in the exchange barrier
+                    pair_bar();                                // every softmax thread takes part in the exchange barriers
+                    pair_bar();
                     if (i >= P_BUFS) mbar_wait(smem_u32(&sm->p_empty[pb]), ((i / P_BUFS) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                     mbar_arrive(smem_u32(&sm->p_full[pb]));
                     return true;
                 }
                 tc_fence_after();
                 float s[HC];
-#pragma unroll
-                for (int c0 = 0; c0 < HC; c0 += 32) {
-                    float t[32];
-                    tc_ld32(tmem_base + TMEM_S + b * BN + half * HC + c0 + lane_off, t);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) s[c0 + j] = t[j];
-                }
+                tc_ld32(tmem_base + TMEM_S + b * BN + half * 64 + grp * HC + lane_off, s);
                 tc_fence_before();
                 mbar_arrive(smem_u32(&sm->s_empty[b]));
-                if (vis != ~0ull) {
+                if (vis != 0xffffffffu) {
 #pragma unroll
-                    for (int j = 0; j < HC; ++j) s[j] = ((vis >> j) & 1ull) ? s[j] : -INFINITY;
+                    for (int j = 0; j < HC; ++j) s[j] = ((vis >> j) & 1u) ? s[j] : -INFINITY;
                 }
                 float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -462,9 +466,10 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                     mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
                 }
                 float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                sm->xch[b][r] = tmax;                          // the partner thread (lane r ^ 64) holds the other 64 keys
+                sm->xch[grp][r] = tmax;                        // the three partner threads hold the other 96 keys of the row
                 pair_bar();
-                tmax = fmaxf(tmax, sm->xch[b][r ^ 64]) * sl2;  // both threads of a row now hold the same value
+                tmax = fmaxf(fmaxf(tmax, sm->xch[grp ^ 1][r]), fmaxf(sm->xch[grp][r ^ 64], sm->xch[grp ^ 1][r ^ 64])) * sl2;
+                pair_bar();                                    // everybody has read: the slots may be written again
                 const bool raise = tmax > m + RAISE || (m == -INFINITY && tmax != -INFINITY);
                 if (__any_sync(0xffffffffu, raise)) {
                     const float f = raise ? ex2_approx(m - tmax) : 1.f;      // m = -inf gives 0
@@ -477,7 +482,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                         mbar_wait(smem_u32(&sm->p_empty[(i - 1) % P_BUFS]), ((i - 1) / P_BUFS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                         tc_fence_after();
 #pragma unroll
-                        for (int c0 = 0; c0 < DH; c0 += 32) {  // this lane's whole row (both threads of a pair scale their copy)
+                        for (int c0 = grp * (DH / 2); c0 < (grp + 1) * (DH / 2); c0 += 32) {  // this lane's row, one half per warp group
                             float v[32];
                             tc_ld32(tmem_base + TMEM_PV + c0 + lane_off, v);
 #pragma unroll
@@ -490,12 +495,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 }
                 const float neg = (m == -INFINITY) ? 0.f : -m;
                 if (i >= P_BUFS) mbar_wait(smem_u32(&sm->p_empty[pb]), ((i / P_BUFS) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
-                // this thread's 64 probabilities are one 128-byte row of key slab `half`; they go into both
+                // this thread's 32 probabilities are half of a 128-byte row of key slab `half`; they go into both
                 // copies of the row (tile rows row and row + 64)
                 uint8_t* prow = p_ptr + pb * P_BYTES + half * (QM * 128) + row * 128;
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
+                for (int q = 0; q < 4; ++q) {
                     uint32_t packed[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -506,7 +511,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                         const __half2 hh = __floats2half2_rn(p0, p1);
                         packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
                     }
-                    const uint32_t off = (uint32_t)((q ^ (row & 7)) << 4);
+                    const uint32_t off = (uint32_t)(((grp * 4 + q) ^ (row & 7)) << 4);
                     const uint4 val = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(prow + off) = val;
                     *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
@@ -516,30 +521,24 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                 return true;
             });
-            float o[HD];
+            float o[OC];
 #pragma unroll
-            for (int c = 0; c < HD; ++c) o[c] = 0.f;
+            for (int c = 0; c < OC; ++c) o[c] = 0.f;
+            const int ocol = half * HD + (HD >= 64 ? grp * OC : 0);      // first output column of this thread
             if (cnt > 0) {
                 // the last product is complete when its P buffer has been released (see the rescale above)
                 mbar_wait(smem_u32(&sm->p_empty[(cnt - 1) % P_BUFS]), ((cnt - 1) / P_BUFS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 if (warp_live) {
                     tc_fence_after();
-#pragma unroll
-                    for (int c0 = 0; c0 < HD; c0 += 32) {
-                        float v[32];
-                        tc_ld32(tmem_base + TMEM_PV + half * HD + c0 + lane_off, v);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) o[c0 + j] = v[j];
-                    }
+                    static_assert(OC == 32, "one 32-column read per thread");
+                    tc_ld32(tmem_base + TMEM_PV + ocol + lane_off, o);
                     tc_fence_before();
                 }
             }
-            pair_bar();                                        // the last exchange of maxima has been read
-            sm->xch[0][r] = l;
+            sm->xch[grp][r] = l;                               // (the exchange slots are free: every unit ends with a barrier)
             pair_bar();
-            l += sm->xch[0][r ^ 64];
-            // all units are done, so the K/V ring is free: it takes the partial
-            leave_partial<DH, HD>(p, split, h, row, half * HD, live, half == 0, o, m, l);
+            l = (l + sm->xch[grp ^ 1][r]) + (sm->xch[grp][r ^ 64] + sm->xch[grp ^ 1][r ^ 64]);
+            leave_partial<DH, OC>(p, split, h, row, ocol, live && carries, half == 0 && grp == 0, o, m, l);
         }
     }
 
@@ -578,7 +577,7 @@ int launch_attn_tc_small(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, cons
     int splits = c->opt_attn_splits;
     if (splits <= 0) {
         splits = c->sm_count / H;                        // one CTA per SM
-        const int by_len = (units + 1) / 2;              // at least two units per split
+        const int by_len = units;                        // at least one unit per split
         if (splits > by_len) splits = by_len;
     }
     if (splits > c->max_splits - (coo ? 1 : 0)) splits = c->max_splits - (coo ? 1 : 0);
