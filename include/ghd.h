@@ -75,9 +75,9 @@ typedef enum ghd_option {
                                  (two groups of four warps on the same tensor-memory lanes), 1 = one thread per row     */
     GHD_OPT_GEMM_SKEW = 14,   /* tcgen05 GEMM with three CTAs per two tiles: k-chunks taken from the middle CTA of every
                                  group (0 = automatic, 1 = none, s + 1 = s chunks), so that it is done before its neighbours */
-    GHD_OPT_ATTN_SMALL = 15,  /* tcgen05 attention, trees of up to 64 nodes: the kernel with 128-key units, four softmax
-                                 threads per query row and the output accumulator resident in tensor memory: 0 = over a
-                                 cache of at least 1024 rows (where it measured faster), 1 = always, 2 = never        */
+    GHD_OPT_ATTN_SMALL = 15,  /* tcgen05 attention: the kernel with 128-key units, four softmax threads per query row and
+                                 the output accumulator resident in tensor memory: 0 = over a cache of at least 1024 rows
+                                 (where it measured faster), 1 = always, 2 = never (64-key units, k_attn_tc)        */
     GHD_OPT_ATTN_SPARSE = 9   /* how the attention handles the new (drafted) keys, the sparse part of
                                  Sec. III-B-3: 0 = packed ancestor bitmask, 64-node groups skipped when
                                  nobody sees them (default); 1 = per-query list of visible nodes (the

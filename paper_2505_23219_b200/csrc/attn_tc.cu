@@ -596,11 +596,12 @@ ghd_status launch_attn_tc(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, con
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: operands must be 16-byte aligned");
         return GHD_EINVAL;
     }
-    // The small-tree kernel (128-key units, four softmax threads per row, accumulator resident in tensor memory): as
-    // measured it wins from about 1024 cache rows on (64 nodes: 19.8 -> 16.8 us at KV 2048, 27.5 -> 22.5 us at KV 4096,
-    // attention + merge) and loses up to 1.5 us on caches of 256 rows.
+    // The kernel with 128-key units, four softmax threads per row and the accumulator resident in tensor memory
+    // (attn_tc_small.cu): as measured it wins from about 1024 cache rows on (attention + merge, 64 nodes: 19.8 -> 16.8 us
+    // at KV 2048, 27.5 -> 22.5 us at KV 4096; 256 nodes: 43.1 -> 36.5 us and 62.0 -> 50.7 us) and is level or up to
+    // 1.5 us behind on caches of 256-512 rows.
     const bool small = c->opt_attn_small == 1 || (c->opt_attn_small == 0 && kv_len_host_of(c, t) >= 1024);
-    if (n <= 64 && small) {
+    if (small) {
         ghd_status st;
         const int s = launch_attn_tc_small(c, q, kv, t, coo, &st);
         if (s <= 0) return st;

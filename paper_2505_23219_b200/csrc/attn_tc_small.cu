@@ -1,9 +1,10 @@
-// Tree attention for trees of up to 64 nodes on the tensor cores (sm_100a, half in, float softmax/accumulate):
-// the small-tree shape of k_attn_tc with 128-key units and the output accumulator kept in tensor memory.
+// Tree attention on the tensor cores (sm_100a, half in, float softmax/accumulate) with 128-key units, four softmax
+// threads per query row and the output accumulator kept in tensor memory: the kernel for long caches.
 //
-// One CTA = one head x one KV split.  FOUR threads share a query row: the queries (at most 64 rows) are loaded
-// twice (tile rows r and r + 64 hold the same query; the copy picks a 64-key half of a unit and a half of d_head)
-// and two groups of four softmax warps work on the same tensor-memory lanes (the group picks 32 of those 64 keys).
+// One CTA = one head x one tile of query rows x one KV split.  FOUR threads share a query row.  Up to 64 nodes
+// (k_attn_small): the queries are loaded twice (tile rows r and r + 64 hold the same query; the copy picks a 64-key
+// half of a unit and a half of d_head) and two groups of four softmax warps work on the same tensor-memory lanes (the
+// group picks 32 of those 64 keys).  More nodes (k_attn_wide): 128 distinct rows per CTA and four such groups.
 // The per-unit softmax work of a thread - one 32-column read of S, 32 exponentials, four 16-byte stores of P - is
 // what the unit chain waits for, so spreading it over 256 threads shortens every unit.
 // Keys are walked in 128-key units: the cache rows [0, kv_len) first (the dense part), then the new rows as one
@@ -33,7 +34,8 @@ namespace {
 using namespace tc;
 
 constexpr int QM = 128;        // query rows per CTA (MMA M)
-constexpr int THREADS = 352;       // producer, S issuer, four softmax warps, PV issuer, four more softmax warps
+constexpr int THREADS_DUP = 352;   // producer, S issuer, four softmax warps, PV issuer, four more softmax warps
+constexpr int THREADS_WIDE = 608;  // ... and eight more: four groups of four softmax warps
 constexpr int MAX_UNITS_WORDS = GHD_MAX_NODES / 64;
 constexpr int NODE_WEIGHT = 2;     // cost of a node-group unit in cache-tile units, for the split of a head
 constexpr int CTRL_BYTES = 1536;   // control block behind the tiles
@@ -83,11 +85,12 @@ struct AttnSmem {
     unsigned long long word_or[MAX_UNITS_WORDS];
     uint32_t tmem_base;
     int abort_flag;
-    float xch[2][QM];             // the four threads of a row exchange their partial maxima and, at the end, sums: [warp group][lane]
+    float xch[2][QM];             // the four threads of a row exchange their partial maxima: float [2][128] when the rows are
+                                  // duplicated, bfloat16 [4][128] (as uint16) when four warp groups share 128 distinct rows
 };
 static_assert(sizeof(AttnSmem) <= CTRL_BYTES, "control block too large");
 
-__device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, 256;" ::: "memory"); }     // all softmax threads
+template <int NT> __device__ __forceinline__ void pair_bar() { asm volatile("bar.sync 2, %0;" ::"n"(NT) : "memory"); }     // all softmax threads
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -114,7 +117,7 @@ __device__ __forceinline__ void leave_partial(const AttnParams& p, int split, in
 // At most 64 query rows.  The queries are loaded twice (tile rows r and r + 64 hold the same query), so S, P and
 // PV come out duplicated and two threads share a row: thread r takes the first 64 keys of a unit and the first
 // half of d_head, thread r + 64 the rest.
-template <int DH>
+template <int DH, bool DUP>
 __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p) {
     using SH = Shape<DH>;
     constexpr int SLABS = SH::SLABS;
@@ -135,6 +138,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y;
+    const int row0 = DUP ? 0 : (int)blockIdx.z * QM;        // first query row of this CTA's tile
+    constexpr int NT = DUP ? 256 : 512;                    // softmax threads
 
     if (threadIdx.x == 32) {        // descriptor fetches overlap the barrier set-up
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
@@ -149,15 +154,15 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sm->s_full[b]), 1);
-            mbar_init(smem_u32(&sm->s_empty[b]), 256);
-            mbar_init(smem_u32(&sm->p_full[b]), 256);
+            mbar_init(smem_u32(&sm->s_empty[b]), NT);
+            mbar_init(smem_u32(&sm->p_full[b]), NT);
             mbar_init(smem_u32(&sm->p_empty[b]), 1);
             mbar_init(smem_u32(&sm->pv_full[b]), 1);
-            mbar_init(smem_u32(&sm->pv_empty[b]), 256);
+            mbar_init(smem_u32(&sm->pv_empty[b]), NT);
         }
         mbar_init(smem_u32(&sm->drain), 1);
         mbar_init(smem_u32(&sm->drain_pv), 1);
-        mbar_init(smem_u32(&sm->mask_ready), 256);
+        mbar_init(smem_u32(&sm->mask_ready), NT);
         for (int w = 0; w < MAX_UNITS_WORDS; ++w) sm->word_or[w] = 0ull;
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -283,9 +288,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 mbar_expect_tx(smem_u32(&sm->q_full), Q_BYTES);
 #pragma unroll
                 for (int s = 0; s < SLABS; ++s) {
-                    // 64-row box, twice: rows 64..127 repeat rows 0..63
-                    tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
-                    tma_load_2d(q_addr + s * Q_SLAB + 64 * 128, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
+                    if constexpr (DUP) {       // 64-row box, twice: rows 64..127 repeat rows 0..63
+                        tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
+                        tma_load_2d(q_addr + s * Q_SLAB + 64 * 128, &tm_q, h * DH + s * 64, 0, smem_u32(&sm->q_full), pol_q);
+                    } else {
+                        tma_load_2d(q_addr + s * Q_SLAB, &tm_q, h * DH + s * 64, row0, smem_u32(&sm->q_full), pol_q);
+                    }
                 }
             }
             while (ok && (more_k || more_v)) {
@@ -389,32 +397,38 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
         }
     } else if ((warp >= 2 && warp <= 5) || warp >= 7) {
         // ------------------------------------------------ softmax warps
-        // FOUR threads per query row.  The tile rows r and r + 64 hold the same query (half = r / 64 picks the 64-key
-        // half of a unit and the half of d_head), and two groups of four warps (warps 2..5 and 7..10) work on the same
-        // tensor-memory lanes (grp picks 32 of those 64 keys and, when the accumulator is rescaled, half of its columns).
+        // FOUR threads per query row, each with 32 of a unit's 128 keys (key block kb).  DUP: the tile rows r and
+        // r + 64 hold the same query and two groups of four warps (warps 2..5 and 7..10) work on the same tensor-memory
+        // lanes: kb = 2 (r / 64) + group.  Otherwise 128 distinct rows and four groups (warps 2..5, 7..10, 11..14,
+        // 15..18): kb = group.  A thread also owns a share of the row's accumulator columns (for the rare rescale and
+        // for carrying the result home): columns [32 cb, 32 cb + 32), cb = its index among the threads of its lane.
         constexpr int HC = 32;                                 // keys of a unit per thread: a quarter of the unit's 128
         static_assert(BN / 4 == HC, "a thread takes 32 keys of a unit");
-        constexpr int HD = DH / 2;                             // d_head columns per row copy
-        constexpr int OC = HD >= 64 ? HD / 2 : HD;             // output columns a thread carries home at the end
-        const int grp = warp >= 7 ? 1 : 0;
-        const bool carries = HD >= 64 || grp == 0;             // (d_head 64: the first group takes all 32 columns of its half)
+        constexpr int NG = DUP ? 2 : 4;                        // warp groups
+        const int grp = warp < 7 ? 0 : 1 + (warp - 7) / 4;
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                        // tensor-memory lane
-        const int half = r >> 6;
-        const int row = r & 63;                                // query row
+        const int kb = DUP ? 2 * (r >> 6) + grp : grp;         // key block
+        const int row = DUP ? (r & 63) : row0 + r;             // query row
+        const int prow_i = DUP ? (r & 63) : r;                 // row of the P tile this thread writes (DUP: and that row + 64)
+        // accumulator columns: DUP - each row copy holds all DH columns, the copy takes a half and the group half of that
+        // (d_head 64: the first group all 32 of the half); otherwise the four groups take DH / 4 each (d_head 64: two groups 32 each)
+        constexpr int CBN = DH / 32;                           // 32-column blocks of a row
+        const int cb = DUP ? (r >> 6) * (CBN / 2) + (CBN >= 4 ? grp : 0) : grp;
+        const bool carries = DUP ? (CBN >= 4 || grp == 0) : grp < CBN;
         const bool live = row < p.n;
-        const bool warp_live = (quad & 1) * 32 < p.n;          // warps whose 32 rows are all padding skip the math
+        const bool warp_live = DUP ? (quad & 1) * 32 < p.n : row0 + quad * 32 < p.n;   // warps whose 32 rows are all padding skip the math
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
         const float sl2 = p.scale * 1.4426950408889634f;       // scores are kept in the log2 domain: s * scale * log2(e)
         pdl_wait();                                            // the mask comes from an earlier kernel
         // this row's mask words stay in registers; their OR over the CTA's rows tells every role
         // which node groups exist for this CTA
-        constexpr int MW = 1;                                  // up to 64 nodes: one mask word (a word that does not exist reads as 0)
+        constexpr int MW = DUP ? 1 : MAX_UNITS_WORDS;          // up to 64 nodes: one mask word (a word that does not exist reads as 0)
         unsigned long long myw[MW];
 #pragma unroll
         for (int w = 0; w < MW; ++w) {
             myw[w] = (live && w < p.n_words) ? p.mask[(size_t)row * p.n_words + w] : 0ull;
-            if (myw[w] && half == 0) atomicOr(&sm->word_or[w], myw[w]);
+            if (myw[w] && kb == 0) atomicOr(&sm->word_or[w], myw[w]);
         }
         mbar_arrive(smem_u32(&sm->mask_ready));
         {
@@ -436,23 +450,25 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 const int b = i & 1, pb = i % P_BUFS;
                 uint32_t vis = 0u;                             // visibility of this thread's 32 keys of the unit
                 if (g < 0) {
-                    const int valid = kv_len - key0 - half * 64 - grp * HC;
+                    const int valid = kv_len - key0 - kb * HC;
                     if (live) vis = valid >= HC ? 0xffffffffu : (valid > 0 ? ((1u << valid) - 1u) : 0u);
-                } else if (g * KSL + half == 0) {
-                    vis = (uint32_t)(myw[0] >> (grp * HC));    // up to 64 nodes: only word 0 exists
+                } else {
+                    const int word = g * KSL + (kb >> 1);      // this thread's 32 nodes of the group: half of a mask word
+#pragma unroll
+                    for (int a = 0; a < MW; ++a) if (a == word) vis = (uint32_t)(myw[a] >> ((kb & 1) * HC));
                 }
                 mbar_wait(smem_u32(&sm->s_full[b]), (i >> 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 if (!warp_live) {
                     mbar_arrive(smem_u32(&sm->s_empty[b]));
-                    pair_bar();                                // every softmax thread takes part in the exchange barriers
-                    pair_bar();
+                    pair_bar<NT>();                                // every softmax thread takes part in the exchange barriers
+                    pair_bar<NT>();
                     if (i >= P_BUFS) mbar_wait(smem_u32(&sm->p_empty[pb]), ((i / P_BUFS) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                     mbar_arrive(smem_u32(&sm->p_full[pb]));
                     return true;
                 }
                 tc_fence_after();
                 float s[HC];
-                tc_ld32(tmem_base + TMEM_S + b * BN + half * 64 + grp * HC + lane_off, s);
+                tc_ld32(tmem_base + TMEM_S + b * BN + kb * HC + lane_off, s);
                 tc_fence_before();
                 mbar_arrive(smem_u32(&sm->s_empty[b]));
                 if (vis != 0xffffffffu) {
@@ -466,10 +482,26 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                     mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
                 }
                 float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                sm->xch[grp][r] = tmax;                        // the three partner threads hold the other 96 keys of the row
-                pair_bar();
-                tmax = fmaxf(fmaxf(tmax, sm->xch[grp ^ 1][r]), fmaxf(sm->xch[grp][r ^ 64], sm->xch[grp ^ 1][r ^ 64])) * sl2;
-                pair_bar();                                    // everybody has read: the slots may be written again
+                // the three partner threads hold the other 96 keys of the row
+                if constexpr (DUP) {
+                    sm->xch[grp][r] = tmax;
+                    pair_bar<NT>();
+                    tmax = fmaxf(fmaxf(tmax, sm->xch[grp ^ 1][r]), fmaxf(sm->xch[grp][r ^ 64], sm->xch[grp ^ 1][r ^ 64])) * sl2;
+                } else {
+                    // Four groups: the maxima travel as bfloat16 (the exchange block holds 1 KB).  Every thread, the owner
+                    // included, uses the ROUNDED values, so all four agree; the reference maximum only has to be common to
+                    // the row and close to the true one (a rounding of 2^-8 relative moves the probabilities by a factor
+                    // near 1, far from the 2^8 head-room).
+                    uint16_t* x16 = reinterpret_cast<uint16_t*>(&sm->xch[0][0]);
+                    x16[grp * QM + r] = (uint16_t)(__float_as_uint(tmax) >> 16);       // truncation: never above the true value...
+                    pair_bar<NT>();
+                    float t4 = -INFINITY;
+#pragma unroll
+                    for (int a = 0; a < NG; ++a) t4 = fmaxf(t4, __uint_as_float((uint32_t)x16[a * QM + r] << 16));
+                    // ... for positive values; a negative one is truncated towards zero, i.e. upwards: both are within 2^-7 relative
+                    tmax = t4 * sl2;
+                }
+                pair_bar<NT>();                                    // everybody has read: the slots may be written again
                 const bool raise = tmax > m + RAISE || (m == -INFINITY && tmax != -INFINITY);
                 if (__any_sync(0xffffffffu, raise)) {
                     const float f = raise ? ex2_approx(m - tmax) : 1.f;      // m = -inf gives 0
@@ -481,13 +513,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                         // unit and is looked at only now and then is not.)
                         mbar_wait(smem_u32(&sm->p_empty[(i - 1) % P_BUFS]), ((i - 1) / P_BUFS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                         tc_fence_after();
-#pragma unroll
-                        for (int c0 = grp * (DH / 2); c0 < (grp + 1) * (DH / 2); c0 += 32) {  // this lane's row, one half per warp group
+                        if (carries) {                         // this thread's own block of the row's columns
                             float v[32];
-                            tc_ld32(tmem_base + TMEM_PV + c0 + lane_off, v);
+                            tc_ld32(tmem_base + TMEM_PV + cb * 32 + lane_off, v);
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] *= f;
-                            tc_st32(tmem_base + TMEM_PV + c0 + lane_off, v);
+                            tc_st32(tmem_base + TMEM_PV + cb * 32 + lane_off, v);
                         }
                         tc_fence_before();
                     }
@@ -497,7 +528,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                 if (i >= P_BUFS) mbar_wait(smem_u32(&sm->p_empty[pb]), ((i / P_BUFS) - 1) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
                 // this thread's 32 probabilities are half of a 128-byte row of key slab `half`; they go into both
                 // copies of the row (tile rows row and row + 64)
-                uint8_t* prow = p_ptr + pb * P_BYTES + half * (QM * 128) + row * 128;
+                uint8_t* prow = p_ptr + pb * P_BYTES + (kb >> 1) * (QM * 128) + prow_i * 128;
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -511,34 +542,34 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
                         const __half2 hh = __floats2half2_rn(p0, p1);
                         packed[e] = *reinterpret_cast<const uint32_t*>(&hh);
                     }
-                    const uint32_t off = (uint32_t)(((grp * 4 + q) ^ (row & 7)) << 4);
+                    const uint32_t off = (uint32_t)((((kb & 1) * 4 + q) ^ (prow_i & 7)) << 4);
                     const uint4 val = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(prow + off) = val;
-                    *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
+                    if constexpr (DUP) *reinterpret_cast<uint4*>(prow + 64 * 128 + off) = val;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(smem_u32(&sm->p_full[pb]));
                 l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                 return true;
             });
-            float o[OC];
+            float o[32];
 #pragma unroll
-            for (int c = 0; c < OC; ++c) o[c] = 0.f;
-            const int ocol = half * HD + (HD >= 64 ? grp * OC : 0);      // first output column of this thread
+            for (int c = 0; c < 32; ++c) o[c] = 0.f;
             if (cnt > 0) {
                 // the last product is complete when its P buffer has been released (see the rescale above)
                 mbar_wait(smem_u32(&sm->p_empty[(cnt - 1) % P_BUFS]), ((cnt - 1) / P_BUFS) & 1, abort_flag, p.status, DEV_TIMEOUT_EPI);
-                if (warp_live) {
+                if (warp_live && carries) {
                     tc_fence_after();
-                    static_assert(OC == 32, "one 32-column read per thread");
-                    tc_ld32(tmem_base + TMEM_PV + ocol + lane_off, o);
+                    tc_ld32(tmem_base + TMEM_PV + cb * 32 + lane_off, o);
                     tc_fence_before();
                 }
             }
-            sm->xch[grp][r] = l;                               // (the exchange slots are free: every unit ends with a barrier)
-            pair_bar();
-            l = (l + sm->xch[grp ^ 1][r]) + (sm->xch[grp][r ^ 64] + sm->xch[grp ^ 1][r ^ 64]);
-            leave_partial<DH, OC>(p, split, h, row, ocol, live && carries, half == 0 && grp == 0, o, m, l);
+            // the four partial sums of a row meet in the P buffers, which nobody reads any more
+            float* lx = reinterpret_cast<float*>(p_ptr);
+            lx[kb * QM + prow_i] = l;
+            pair_bar<NT>();
+            l = (lx[prow_i] + lx[QM + prow_i]) + (lx[2 * QM + prow_i] + lx[3 * QM + prow_i]);
+            leave_partial<DH, 32>(p, split, h, row, cb * 32, live && carries, kb == 0, o, m, l);
         }
     }
 
@@ -551,9 +582,16 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& tm_q, const CUtenso
 }
 
 template <int DH>
-__global__ void __launch_bounds__(THREADS, 1) k_attn_small(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                                                           const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
-    attn_body<DH>(tm_q, tm_k, tm_v, p);
+__global__ void __launch_bounds__(THREADS_DUP, 1) k_attn_small(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                                                               const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    attn_body<DH, true>(tm_q, tm_k, tm_v, p);
+}
+
+// The same kernel for trees of more than 64 nodes: 128 distinct query rows per CTA, four groups of softmax warps.
+template <int DH>
+__global__ void __launch_bounds__(THREADS_WIDE, 1) k_attn_wide(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                                                               const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    attn_body<DH, false>(tm_q, tm_k, tm_v, p);
 }
 
 }  // namespace
@@ -566,17 +604,19 @@ int launch_attn_tc_small(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, cons
     const int kt = t->kv_len < 0 ? m.max_kv_len : t->kv_len + n;      // rows the K/V maps cover (see launch_attn_tc)
     *st = GHD_OK;
     CUtensorMap tm_q, tm_k, tm_v;
-    if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, 64, &tm_q) ||
+    const bool dup = n <= 64;                            // duplicated rows (two warp groups) or 128 distinct rows (four)
+    const int mtiles = (n + QM - 1) / QM;
+    if (!tmap_rows_x_k(c, q, (uint64_t)n, (uint64_t)d, dup ? 64 : QM, &tm_q) ||
         !tmap_planes_slabs(c, kv->k, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, (uint32_t)BN, &tm_k) ||
         !tmap_planes_slabs(c, kv->v, (uint64_t)H, (uint64_t)m.max_kv_len, (uint64_t)kt, (uint64_t)dh, (uint32_t)BN, &tm_v)) {
         snprintf(c->err, sizeof(c->err), "tcgen05 attention: tensor map encoding failed");
         *st = GHD_ECUDA;
         return 0;
     }
-    const int units = (kv_len_host_of(c, t) + BN - 1) / BN + (coo ? 0 : 1);
+    const int units = (kv_len_host_of(c, t) + BN - 1) / BN + (coo ? 0 : (n + BN - 1) / BN);
     int splits = c->opt_attn_splits;
     if (splits <= 0) {
-        splits = c->sm_count / H;                        // one CTA per SM
+        splits = c->sm_count / (H * mtiles);             // one CTA per SM
         const int by_len = units;                        // at least one unit per split
         if (splits > by_len) splits = by_len;
     }
@@ -587,10 +627,12 @@ int launch_attn_tc_small(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, cons
     p.max_nodes = m.max_nodes; p.splits = splits; p.n_words = t->n_words; p.cache_only = coo ? 1 : 0;
     p.mask = t->mask; p.status = c->status; p.part_o = c->att_o; p.part_ml = c->att_ml;
     p.scale = 1.0f / sqrtf((float)dh);
-    dim3 grid(splits, H, 1);
+    dim3 grid(splits, H, mtiles);
     if (!c->attr_attn_small) {       // per context: the attribute belongs to the device the context was created on
         if (cudaFuncSetAttribute(k_attn_small<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Shape<64>::SMEM_BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(k_attn_small<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Shape<128>::SMEM_BYTES) != cudaSuccess) {
+            cudaFuncSetAttribute(k_attn_small<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Shape<128>::SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_wide<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Shape<64>::SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_wide<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Shape<128>::SMEM_BYTES) != cudaSuccess) {
             snprintf(c->err, sizeof(c->err), "tcgen05 attention: cannot raise dynamic shared memory");
             cudaGetLastError();
             *st = GHD_ECUDA;
@@ -598,8 +640,13 @@ int launch_attn_tc_small(ghd_ctx* c, const void* q, const ghd_kv_layer* kv, cons
         }
         c->attr_attn_small = true;
     }
-    if (dh == 64) launch_k(c, true, k_attn_small<64>, grid, THREADS, Shape<64>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
-    else launch_k(c, true, k_attn_small<128>, grid, THREADS, Shape<128>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
+    if (dup) {
+        if (dh == 64) launch_k(c, true, k_attn_small<64>, grid, THREADS_DUP, Shape<64>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
+        else launch_k(c, true, k_attn_small<128>, grid, THREADS_DUP, Shape<128>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
+    } else {
+        if (dh == 64) launch_k(c, true, k_attn_wide<64>, grid, THREADS_WIDE, Shape<64>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
+        else launch_k(c, true, k_attn_wide<128>, grid, THREADS_WIDE, Shape<128>::SMEM_BYTES, tm_q, tm_k, tm_v, p);
+    }
     return splits;
 }
 

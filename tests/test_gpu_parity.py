@@ -290,6 +290,19 @@ def test_tree_attention_small_tree_kernel_with_128_key_units(ghd, shape, n, L, s
     assert _attention_case(ghd, wl.scaled(shape, name="chain"), n, L, wl.chain_tree(n), splits, opts=small) <= 2e-3
 
 
+@pytest.mark.parametrize("shape", [SMALL16, SMALL16_DH128], ids=["f16", "f16dh128"])
+@pytest.mark.parametrize("n,L,splits", [(65, 0, 0), (100, 300, 0), (128, 1000, 3), (130, 17, 2), (200, 1000, 0), (256, 129, 0), (256, 2048, 0),
+                                        (256, 4096, 2), (129, 127, 1)])
+def test_tree_attention_128_key_unit_kernel_on_wide_trees(ghd, shape, n, L, splits):
+    """The same kernel on 128 distinct query rows per CTA with four groups of softmax warps (GHD_OPT_ATTN_SMALL = 1)."""
+    parent = wl.random_tree(n, 8, 1000 + n, max_children=6)
+    wide = [(ghd.OPT_ATTN_SMALL, 1)]
+    assert _attention_case(ghd, shape, n, L, parent, splits, opts=wide) <= 2e-3
+    assert _attention_case(ghd, shape, n, L, parent, splits, sparse=1, opts=wide) <= 2e-3
+    assert _attention_case(ghd, shape, n, L, parent, splits, on_device=True, opts=wide) <= 2e-3
+    assert _attention_case(ghd, shape, n, L, wl.star_tree(n), splits, opts=wide) <= 2e-3
+
+
 @pytest.mark.parametrize("n,L", [(1, 40), (13, 100), (64, 77)])
 def test_small_layers_with_the_small_tree_attention_kernel(ghd, n, L):
     import paper_2505_23219_b200 as g
